@@ -1,0 +1,184 @@
+/*
+ * wfq.h - C ABI of the group-wise int8-quantized Winograd convolution F(m,3) for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates y = conv2d(x, w, stride 1, padding 1, no bias) (deep-learning
+ * cross-correlation) for 3x3 filters through the quantized Winograd pipeline of the
+ * paper "Data-Free Group-Wise Fully Quantized Winograd Convolution via Learnable
+ * Scales" (Section 3.1 for the algorithm, Section 4.1 for the scaled transforms and
+ * the quantized Hadamard stage, Eq. quant-Y):
+ *
+ *   W = S_G V_G w V_G^T S_G        filter transform, offline        (wfq_prepare_filters)
+ *   X = S_B V_B x V_B^T S_B        input transform, fp32
+ *   Xq, sX = Q(X)                  int8 codes + one fp32 scale per group of
+ *                                  `group_size` consecutive input channels, per
+ *                                  Winograd position and tile (dynamic abs-max)
+ *   acc[g] = sum_{c in g} Xq Wq    int8 x int8 -> int32 on the tensor cores,
+ *                                  one matrix product per Winograd position
+ *   Y = sum_g acc[g] sX[g] sW[g]   per-group dequantization into fp32
+ *   y = V_A S_A Y S_A V_A^T        output transform, fp32, cropped to H x W
+ *
+ * Notation: n = m + 2, P = n*n positions (p = i*n + j), TH = ceil(H/m),
+ * TW = ceil(W/m), T = N*TH*TW tiles (t = (img*TH + th)*TW + tw), G = C/group_size.
+ *
+ * Quantizer (per group, fp32): amax = max|v|; if amax < 1e-30 the scale is 0 and all
+ * codes are 0; otherwise scale = amax/127, inv = 127/amax (both correctly rounded) and
+ * code = clamp(round_half_even(v*inv), -127, 127).
+ *
+ * General rules
+ *   - All functions return a wfq_status_t; nothing throws, aborts or traps.
+ *   - Arguments are validated before any device work is launched.
+ *   - "device" pointers are CUDA device pointers of the current device, "host"
+ *     pointers are ordinary host memory.  `stream` is a cudaStream_t passed as void*
+ *     (NULL = the default stream).
+ *   - Work is asynchronous on `stream` unless stated; buffers must stay valid until
+ *     that work has completed.  One plan must not be used from two threads or two
+ *     streams at the same time (its workspace is shared).
+ *   - The library needs a device of compute capability 10.x; on anything else the
+ *     launching calls return WFQ_ERR_UNSUPPORTED or WFQ_ERR_CUDA.  There is no CPU
+ *     fallback.
+ */
+#ifndef WFQ_H_
+#define WFQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct wfq_plan wfq_plan_t; /* opaque, owned by the library */
+
+typedef enum {
+    WFQ_OK = 0,
+    WFQ_ERR_INVALID_ARG = 1,  /* NULL pointer, non-positive size, bad enum value */
+    WFQ_ERR_UNSUPPORTED = 2,  /* valid request outside the supported set */
+    WFQ_ERR_ALLOC = 3,        /* host or device allocation failed */
+    WFQ_ERR_NOT_PREPARED = 4, /* workspace or filters missing */
+    WFQ_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed */
+    WFQ_ERR_TIMEOUT = 6       /* a bounded device-side wait expired (status word) */
+} wfq_status_t;
+
+typedef enum { WFQ_F32 = 0, WFQ_F16 = 1 } wfq_dtype_t;
+
+/* Buffers that wfq_debug_get can expose (all device memory). */
+typedef enum {
+    WFQ_BUF_XQ = 0,     /* int8  Xq[P][T][C]            (workspace)  */
+    WFQ_BUF_SX = 1,     /* fp32  sX[P][G][T]            (workspace)  */
+    WFQ_BUF_WQ = 2,     /* int8  Wq[P][K][C]            (plan-owned) */
+    WFQ_BUF_SW = 3,     /* fp32  sW[P][G][K]            (plan-owned) */
+    WFQ_BUF_Y = 4,      /* fp32  Y[P][K][Tp], Tp = T rounded up to 32 (workspace) */
+    WFQ_BUF_STATUS = 5  /* int32 status[4]: {code, where, block, aux} (plan-owned) */
+} wfq_buffer_t;
+
+/*
+ * Create a plan for one layer: x[N][C][H][W] -> y[N][K][H][W] evaluated as F(m,3)
+ * (Section 3.1: output tile m x m, filter r x r, input tile (m+r-1)^2).
+ * Supported: r = 3; m in {4, 6}; bits = 8; group_size a multiple of 32, at most 256,
+ * dividing C; N, C, K, H, W >= 1; P*T*C, P*K*C and N*K*H*W below 2^31.
+ * Returns WFQ_ERR_INVALID_ARG for NULL/non-positive arguments and
+ * WFQ_ERR_UNSUPPORTED for anything else outside this set.  Synchronous, host-only
+ * (no device is touched).
+ */
+wfq_status_t wfq_plan_create(wfq_plan_t **out, int N, int C, int K, int H, int W, int m,
+                             int r, int group_size, int bits);
+
+/* Element type of x in wfq_conv_forward (default WFQ_F32).  Call before forward. */
+wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype);
+
+/*
+ * Bytes of caller-owned device scratch the plan needs (Xq + sX + Y, each region
+ * 1024-byte aligned).  Returns 0 for a NULL plan.
+ */
+size_t wfq_plan_workspace_bytes(const wfq_plan_t *plan);
+
+/*
+ * Hand the plan its scratch memory: `dev_ptr` device memory, 1024-byte aligned, at
+ * least wfq_plan_workspace_bytes() long, owned by the caller and kept alive while the
+ * plan is used.  Builds the TMA descriptor of Xq.  WFQ_ERR_INVALID_ARG if too small or
+ * misaligned.
+ */
+wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t bytes);
+
+/*
+ * Offline filter path (Section 4.1, W = S_G V_G w V_G^T S_G; "weight transformation can
+ * be done offline with high precision"): transform in fp64, round once to fp32,
+ * quantize every group of `group_size` consecutive input channels per (position,
+ * output channel), and store the codes position-major (the paper's offline reordering
+ * of weights to compute order).
+ *   w_dev    device, fp32 [K][C][3][3]
+ *   sB_host  host, n floats, diagonal of S_B (NULL = standard scales of the paper)
+ *   sG_host  host, n floats, diagonal of S_G (NULL = standard scales)
+ *   sA_host  host, n floats, diagonal of S_A (NULL = 1/(sB*sG), Eq. scaling_condition,
+ *            evaluated in fp64 and rounded to fp32)
+ * All scales must be finite and nonzero (signs are allowed).  Allocates the
+ * plan-owned Wq/sW buffers on first use (cudaMalloc), runs on `stream`, and may be
+ * called again to replace the filters.
+ */
+wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const float *sB_host,
+                                 const float *sG_host, const float *sA_host, void *stream);
+
+/*
+ * The hot path: input transform + group quantization, per-position int8 tensor-core
+ * contraction with per-group dequantization, output transform.
+ *   x_dev  device, [N][C][H][W] in the plan's input dtype, 4-byte aligned
+ *   y_dev  device, fp32 [N][K][H][W], 16-byte aligned
+ * Three kernels are enqueued on `stream`; no host synchronisation.  Requires a
+ * workspace and prepared filters (WFQ_ERR_NOT_PREPARED otherwise).
+ */
+wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev, void *stream);
+
+/*
+ * Same computation with HOST buffers: copies x to the device, runs the three kernels,
+ * copies y back, all on `stream`, then waits for the stream (synchronous).  The plan
+ * allocates device staging for x and y on first use.  x_host/y_host should be pinned
+ * for full copy speed.
+ */
+wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *y_host,
+                                   void *stream);
+
+/* The three stages of wfq_conv_forward, separately (tests and profiling). */
+/* Stage 1 (X = S_B V_B x V_B^T S_B, then Q): x_dev -> workspace Xq, sX. */
+wfq_status_t wfq_input_transform_quantize(wfq_plan_t *plan, const void *x_dev, void *stream);
+/* Stage 2 (Eq. quant-Y): workspace Xq, sX and the plan's Wq, sW -> workspace Y. */
+wfq_status_t wfq_gemm_dequantize(wfq_plan_t *plan, void *stream);
+/* Stage 3 (y = V_A S_A Y S_A V_A^T): workspace Y -> y_dev. */
+wfq_status_t wfq_output_transform(wfq_plan_t *plan, float *y_dev, void *stream);
+
+/*
+ * Raw int32 group accumulators of stage 2, before any scaling:
+ *   acc_dev[p][t][k][g] = sum_{c in group g} Xq[p][t][c] * Wq[p][k][c]
+ * computed by the same tensor-core kernel as wfq_gemm_dequantize from the operands
+ * currently in the workspace (Xq) and the plan (Wq).  acc_dev: device, int32,
+ * P*T*K*G elements.
+ */
+wfq_status_t wfq_debug_gemm_acc32(wfq_plan_t *plan, int32_t *acc_dev, void *stream);
+
+/*
+ * Device address and size of an internal buffer (see wfq_buffer_t for layouts).
+ * Tests read intermediates from these and may overwrite the workspace ones to feed a
+ * later stage with chosen operands.
+ */
+wfq_status_t wfq_debug_get(wfq_plan_t *plan, wfq_buffer_t which, void **dev_ptr, size_t *bytes);
+
+/*
+ * Read (synchronously, after waiting for `stream`) the device status word that the
+ * kernels set when one of their bounded waits expires.  Returns WFQ_OK or
+ * WFQ_ERR_TIMEOUT; `where` (may be NULL) receives an identifier of the wait.
+ */
+wfq_status_t wfq_check_device_status(wfq_plan_t *plan, void *stream, int *where);
+
+/* Release the plan and everything it owns (not the workspace).  NULL is accepted. */
+wfq_status_t wfq_plan_destroy(wfq_plan_t *plan);
+
+/* Static string for a status code. */
+const char *wfq_status_string(wfq_status_t status);
+
+/* Library version as major*100 + minor. */
+int wfq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WFQ_H_ */

@@ -1,0 +1,337 @@
+// C ABI of libwfq.so: plan management, argument checks, workspace layout, launch order.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "wfq_internal.h"
+
+namespace {
+
+// Standard scale vectors of the paper's supplementary ("Standard Winograd
+// transforms"): used when the caller passes NULL, and as the reference the kernels'
+// hard-coded integer/rational transform matrices are scaled by.
+const double kStdSB4[6] = {4.0, -6.0, -6.0, 24.0, 24.0, 1.0};
+const double kStdSG4[6] = {1.0 / 4, -1.0 / 6, -1.0 / 6, 1.0 / 24, 1.0 / 24, 1.0};
+const double kStdSB6[8] = {1.0, -4.5, -4.5, 90.0, 90.0, 45.0 / 32, 45.0 / 32, 1.0};
+const double kStdSG6[8] = {1.0, -2.0 / 9, -2.0 / 9, 1.0 / 90, 1.0 / 90, 32.0 / 45, 32.0 / 45, 1.0};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+cudaStream_t as_stream(void *s) { return reinterpret_cast<cudaStream_t>(s); }
+
+wfq_status_t cuda_status(cudaError_t e)
+{
+    if (e == cudaSuccess) return WFQ_OK;
+    if (e == cudaErrorMemoryAllocation) return WFQ_ERR_ALLOC;
+    return WFQ_ERR_CUDA;
+}
+
+wfq_status_t ready_to_run(const wfq_plan *plan)
+{
+    if (!plan) return WFQ_ERR_INVALID_ARG;
+    if (!plan->has_workspace || !plan->prepared) return WFQ_ERR_NOT_PREPARED;
+    return WFQ_OK;
+}
+
+size_t in_elem_bytes(const wfq_plan *plan) { return plan->in_dtype == WFQ_F16 ? 2 : 4; }
+
+}  // namespace
+
+namespace wfq {
+
+bool encode_tmap_bytes3d(CUtensorMap *map, const void *base, int inner, int rows, int planes,
+                         int box_rows)
+{
+    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                 const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                 const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) !=
+                cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+            return false;
+        encode = reinterpret_cast<EncodeFn>(fn);
+    }
+    cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)planes};
+    cuuint64_t strides[2] = {(cuuint64_t)inner, (cuuint64_t)inner * (cuuint64_t)rows};
+    cuuint32_t box[3] = {128u, (cuuint32_t)box_rows, 1u};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace wfq
+
+extern "C" {
+
+int wfq_version(void) { return 100; }
+
+const char *wfq_status_string(wfq_status_t s)
+{
+    switch (s) {
+        case WFQ_OK: return "ok";
+        case WFQ_ERR_INVALID_ARG: return "invalid argument";
+        case WFQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case WFQ_ERR_ALLOC: return "allocation failed";
+        case WFQ_ERR_NOT_PREPARED: return "plan has no workspace or no prepared filters";
+        case WFQ_ERR_CUDA: return "CUDA call failed";
+        case WFQ_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+wfq_status_t wfq_plan_create(wfq_plan_t **out, int N, int C, int K, int H, int W, int m, int r,
+                             int group_size, int bits)
+{
+    if (!out) return WFQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (N < 1 || C < 1 || K < 1 || H < 1 || W < 1 || m < 1 || r < 1 || group_size < 1 || bits < 1)
+        return WFQ_ERR_INVALID_ARG;
+    if (r != 3 || (m != 4 && m != 6) || bits != 8) return WFQ_ERR_UNSUPPORTED;
+    if (group_size % 32 != 0 || group_size > 256 || C % group_size != 0)
+        return WFQ_ERR_UNSUPPORTED;
+
+    wfq_plan *p = new (std::nothrow) wfq_plan();
+    if (!p) return WFQ_ERR_ALLOC;
+    wfq::Geometry &g = p->geo;
+    g.N = N; g.C = C; g.K = K; g.H = H; g.W = W;
+    g.m = m; g.n = m + 2; g.P = g.n * g.n;
+    g.TH = (H + m - 1) / m; g.TW = (W + m - 1) / m;
+    const long long T = (long long)N * g.TH * g.TW;
+    const long long lim = (1LL << 31) - 1;
+    if (T > lim || (long long)g.P * T * C > lim || (long long)g.P * K * C > lim ||
+        (long long)N * K * H * W > lim || (long long)N * C * H * W > lim ||
+        (long long)g.P * K * ((T + 31) / 32 * 32) > lim) {
+        delete p;
+        return WFQ_ERR_UNSUPPORTED;
+    }
+    g.T = (int)T; g.Tp = (g.T + 31) / 32 * 32;
+    g.gs = group_size; g.G = C / group_size;
+
+    wfq::Workspace &ws = p->ws;
+    ws.xq_bytes = align_up((size_t)g.P * g.T * g.C, 1024);
+    ws.sx_bytes = align_up((size_t)g.P * g.G * g.T * sizeof(float), 1024);
+    ws.y_bytes = align_up((size_t)g.P * g.K * g.Tp * sizeof(float), 1024);
+    ws.total = ws.xq_bytes + ws.sx_bytes + ws.y_bytes;
+    *out = p;
+    return WFQ_OK;
+}
+
+wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype)
+{
+    if (!plan) return WFQ_ERR_INVALID_ARG;
+    if (dtype != WFQ_F32 && dtype != WFQ_F16) return WFQ_ERR_INVALID_ARG;
+    plan->in_dtype = dtype;
+    return WFQ_OK;
+}
+
+size_t wfq_plan_workspace_bytes(const wfq_plan_t *plan) { return plan ? plan->ws.total : 0; }
+
+wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t bytes)
+{
+    if (!plan || !dev_ptr) return WFQ_ERR_INVALID_ARG;
+    if (bytes < plan->ws.total || (reinterpret_cast<uintptr_t>(dev_ptr) & 1023u) != 0)
+        return WFQ_ERR_INVALID_ARG;
+    wfq::Workspace &ws = plan->ws;
+    char *base = static_cast<char *>(dev_ptr);
+    ws.Xq = reinterpret_cast<int8_t *>(base);
+    ws.sX = reinterpret_cast<float *>(base + ws.xq_bytes);
+    ws.Y = reinterpret_cast<float *>(base + ws.xq_bytes + ws.sx_bytes);
+    const wfq::Geometry &g = plan->geo;
+    plan->tmap_xq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_xq, ws.Xq, g.C, g.T, g.P,
+                                               wfq::gemm_block_m());
+    if (!plan->tmap_xq_ok) return WFQ_ERR_CUDA;
+    plan->has_workspace = true;
+    return WFQ_OK;
+}
+
+wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const float *sB_host,
+                                 const float *sG_host, const float *sA_host, void *stream)
+{
+    if (!plan || !w_dev) return WFQ_ERR_INVALID_ARG;
+    const wfq::Geometry &g = plan->geo;
+    const double *stdB = g.m == 4 ? kStdSB4 : kStdSB6;
+    const double *stdG = g.m == 4 ? kStdSG4 : kStdSG6;
+    for (int i = 0; i < g.n; ++i) {
+        const double b = sB_host ? (double)sB_host[i] : stdB[i];
+        const double s = sG_host ? (double)sG_host[i] : stdG[i];
+        if (!std::isfinite(b) || !std::isfinite(s) || b == 0.0 || s == 0.0)
+            return WFQ_ERR_INVALID_ARG;
+        double a;
+        if (sA_host) {
+            a = (double)sA_host[i];
+            if (!std::isfinite(a) || a == 0.0) return WFQ_ERR_INVALID_ARG;
+        } else {
+            a = (double)(float)(1.0 / (b * s));
+        }
+        plan->sB[i] = b; plan->sG[i] = s; plan->sA[i] = a;
+    }
+    for (int i = 0; i < g.n; ++i)
+        for (int j = 0; j < g.n; ++j) {
+            plan->tables.in_scale[i * g.n + j] =
+                (float)((plan->sB[i] / stdB[i]) * (plan->sB[j] / stdB[j]));
+            plan->tables.out_scale[i * g.n + j] = (float)(plan->sA[i] * plan->sA[j]);
+        }
+
+    cudaError_t e = cudaGetDevice(&plan->device);
+    if (e != cudaSuccess) return WFQ_ERR_CUDA;
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, plan->device);
+    if (e != cudaSuccess) return WFQ_ERR_CUDA;
+    if (prop.major != 10) return WFQ_ERR_UNSUPPORTED;
+    plan->sm_count = prop.multiProcessorCount;
+
+    const size_t wq_bytes = (size_t)g.P * g.K * g.C;
+    const size_t sw_bytes = (size_t)g.P * g.G * g.K * sizeof(float);
+    if (!plan->Wq && (e = cudaMalloc(&plan->Wq, wq_bytes)) != cudaSuccess) return cuda_status(e);
+    if (!plan->sW && (e = cudaMalloc(&plan->sW, sw_bytes)) != cudaSuccess) return cuda_status(e);
+    if (!plan->status) {
+        if ((e = cudaMalloc(&plan->status, 4 * sizeof(int))) != cudaSuccess) return cuda_status(e);
+        if ((e = cudaMemsetAsync(plan->status, 0, 4 * sizeof(int), as_stream(stream))) != cudaSuccess)
+            return WFQ_ERR_CUDA;
+    }
+    float *w32 = nullptr;  // fp32 transformed filters, released after quantization
+    if ((e = cudaMalloc(&w32, wq_bytes * sizeof(float))) != cudaSuccess) return cuda_status(e);
+    e = wfq::launch_filter_prep(*plan, w_dev, w32, as_stream(stream));
+    cudaError_t e2 = cudaStreamSynchronize(as_stream(stream));
+    cudaFree(w32);
+    if (e != cudaSuccess || e2 != cudaSuccess) return WFQ_ERR_CUDA;
+
+    plan->tmap_wq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_wq, plan->Wq, g.C, g.K, g.P,
+                                               wfq::gemm_block_n());
+    if (!plan->tmap_wq_ok) return WFQ_ERR_CUDA;
+    plan->prepared = true;
+    return WFQ_OK;
+}
+
+wfq_status_t wfq_input_transform_quantize(wfq_plan_t *plan, const void *x_dev, void *stream)
+{
+    wfq_status_t s = ready_to_run(plan);
+    if (s != WFQ_OK) return s;
+    if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 3u)) return WFQ_ERR_INVALID_ARG;
+    return cuda_status(wfq::launch_input_transform(*plan, x_dev, as_stream(stream)));
+}
+
+wfq_status_t wfq_gemm_dequantize(wfq_plan_t *plan, void *stream)
+{
+    wfq_status_t s = ready_to_run(plan);
+    if (s != WFQ_OK) return s;
+    return cuda_status(wfq::launch_gemm(*plan, nullptr, as_stream(stream)));
+}
+
+wfq_status_t wfq_debug_gemm_acc32(wfq_plan_t *plan, int32_t *acc_dev, void *stream)
+{
+    wfq_status_t s = ready_to_run(plan);
+    if (s != WFQ_OK) return s;
+    if (!acc_dev) return WFQ_ERR_INVALID_ARG;
+    return cuda_status(wfq::launch_gemm(*plan, acc_dev, as_stream(stream)));
+}
+
+wfq_status_t wfq_output_transform(wfq_plan_t *plan, float *y_dev, void *stream)
+{
+    wfq_status_t s = ready_to_run(plan);
+    if (s != WFQ_OK) return s;
+    if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 15u)) return WFQ_ERR_INVALID_ARG;
+    return cuda_status(wfq::launch_output_transform(*plan, y_dev, as_stream(stream)));
+}
+
+wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev, void *stream)
+{
+    wfq_status_t s = ready_to_run(plan);
+    if (s != WFQ_OK) return s;
+    if (!x_dev || !y_dev || (reinterpret_cast<uintptr_t>(x_dev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(y_dev) & 15u))
+        return WFQ_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    cudaError_t e = wfq::launch_input_transform(*plan, x_dev, st);
+    if (e == cudaSuccess) e = wfq::launch_gemm(*plan, nullptr, st);
+    if (e == cudaSuccess) e = wfq::launch_output_transform(*plan, y_dev, st);
+    return cuda_status(e);
+}
+
+wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *y_host,
+                                   void *stream)
+{
+    wfq_status_t s = ready_to_run(plan);
+    if (s != WFQ_OK) return s;
+    if (!x_host || !y_host) return WFQ_ERR_INVALID_ARG;
+    const wfq::Geometry &g = plan->geo;
+    const size_t xb = (size_t)g.N * g.C * g.H * g.W * in_elem_bytes(plan);
+    const size_t yb = (size_t)g.N * g.K * g.H * g.W * sizeof(float);
+    cudaError_t e;
+    if (!plan->x_stage && (e = cudaMalloc(&plan->x_stage, (size_t)g.N * g.C * g.H * g.W * 4)) != cudaSuccess)
+        return cuda_status(e);
+    if (!plan->y_stage && (e = cudaMalloc(&plan->y_stage, yb)) != cudaSuccess) return cuda_status(e);
+    cudaStream_t st = as_stream(stream);
+    if ((e = cudaMemcpyAsync(plan->x_stage, x_host, xb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return WFQ_ERR_CUDA;
+    s = wfq_conv_forward(plan, plan->x_stage, plan->y_stage, stream);
+    if (s != WFQ_OK) return s;
+    if ((e = cudaMemcpyAsync(y_host, plan->y_stage, yb, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return WFQ_ERR_CUDA;
+    return cuda_status(cudaStreamSynchronize(st));
+}
+
+wfq_status_t wfq_debug_get(wfq_plan_t *plan, wfq_buffer_t which, void **dev_ptr, size_t *bytes)
+{
+    if (!plan || !dev_ptr || !bytes) return WFQ_ERR_INVALID_ARG;
+    const wfq::Geometry &g = plan->geo;
+    *dev_ptr = nullptr;
+    *bytes = 0;
+    switch (which) {
+        case WFQ_BUF_XQ:
+            if (!plan->has_workspace) return WFQ_ERR_NOT_PREPARED;
+            *dev_ptr = plan->ws.Xq; *bytes = (size_t)g.P * g.T * g.C; return WFQ_OK;
+        case WFQ_BUF_SX:
+            if (!plan->has_workspace) return WFQ_ERR_NOT_PREPARED;
+            *dev_ptr = plan->ws.sX; *bytes = (size_t)g.P * g.G * g.T * sizeof(float); return WFQ_OK;
+        case WFQ_BUF_Y:
+            if (!plan->has_workspace) return WFQ_ERR_NOT_PREPARED;
+            *dev_ptr = plan->ws.Y; *bytes = (size_t)g.P * g.K * g.Tp * sizeof(float); return WFQ_OK;
+        case WFQ_BUF_WQ:
+            if (!plan->prepared) return WFQ_ERR_NOT_PREPARED;
+            *dev_ptr = plan->Wq; *bytes = (size_t)g.P * g.K * g.C; return WFQ_OK;
+        case WFQ_BUF_SW:
+            if (!plan->prepared) return WFQ_ERR_NOT_PREPARED;
+            *dev_ptr = plan->sW; *bytes = (size_t)g.P * g.G * g.K * sizeof(float); return WFQ_OK;
+        case WFQ_BUF_STATUS:
+            if (!plan->status) return WFQ_ERR_NOT_PREPARED;
+            *dev_ptr = plan->status; *bytes = 4 * sizeof(int); return WFQ_OK;
+    }
+    return WFQ_ERR_INVALID_ARG;
+}
+
+wfq_status_t wfq_check_device_status(wfq_plan_t *plan, void *stream, int *where)
+{
+    if (!plan) return WFQ_ERR_INVALID_ARG;
+    if (!plan->status) return WFQ_ERR_NOT_PREPARED;
+    int host[4] = {0, 0, 0, 0};
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemcpyAsync(host, plan->status, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return WFQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return WFQ_ERR_CUDA;
+    if (where) *where = host[1];
+    return host[0] == 0 ? WFQ_OK : WFQ_ERR_TIMEOUT;
+}
+
+wfq_status_t wfq_plan_destroy(wfq_plan_t *plan)
+{
+    if (!plan) return WFQ_OK;
+    if (plan->Wq) cudaFree(plan->Wq);
+    if (plan->sW) cudaFree(plan->sW);
+    if (plan->status) cudaFree(plan->status);
+    if (plan->x_stage) cudaFree(plan->x_stage);
+    if (plan->y_stage) cudaFree(plan->y_stage);
+    delete plan;
+    return WFQ_OK;
+}
+
+}  // extern "C"

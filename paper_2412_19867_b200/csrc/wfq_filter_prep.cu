@@ -1,0 +1,111 @@
+// Offline filter path: W = S_G V_G w V_G^T S_G (Section 4.1) in fp64, one rounding to
+// fp32, then group-wise int8 quantization along the input channels, stored
+// position-major Wq[P][K][C] with scales sW[P][G][K].  Not on the timed path.
+#include "wfq_internal.h"
+
+namespace wfq {
+namespace {
+
+struct GScales {
+    double s[kMaxN];
+};
+
+// Rows of V_{n x 3}: (f^0 g^2, f^1 g^1, f^2 g^0) for the points
+// 0, 1, -1, 2, -2, [1/2, -1/2,] infinity.
+__device__ __forceinline__ void vg_row(int m, int i, double &a, double &b, double &c)
+{
+    const int n = m + 2;
+    if (i == n - 1) { a = 0.0; b = 0.0; c = 1.0; return; }
+    double f;
+    switch (i) {
+        case 0: f = 0.0; break;
+        case 1: f = 1.0; break;
+        case 2: f = -1.0; break;
+        case 3: f = 2.0; break;
+        case 4: f = -2.0; break;
+        case 5: f = 0.5; break;
+        default: f = -0.5; break;
+    }
+    a = 1.0; b = f; c = f * f;
+}
+
+// One thread per (k, c): all P transformed values, rounded to fp32.
+__global__ void filter_transform_kernel(const float *__restrict__ w, float *__restrict__ w32,
+                                        int K, int C, int m, GScales sg)
+{
+    const int n = m + 2;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)K * C) return;
+    const int c = (int)(idx % C), k = (int)(idx / C);
+    double f[9];
+    for (int i = 0; i < 9; ++i) f[i] = (double)w[idx * 9 + i];
+    double tmp[kMaxN][3];  // V_G w
+    for (int i = 0; i < n; ++i) {
+        double a, b, cc;
+        vg_row(m, i, a, b, cc);
+        for (int col = 0; col < 3; ++col)
+            tmp[i][col] = a * f[col] + b * f[3 + col] + cc * f[6 + col];
+    }
+    for (int i = 0; i < n; ++i)
+        for (int j = 0; j < n; ++j) {
+            double a, b, cc;
+            vg_row(m, j, a, b, cc);
+            const double u = tmp[i][0] * a + tmp[i][1] * b + tmp[i][2] * cc;
+            w32[((size_t)(i * n + j) * K + k) * C + c] = (float)(sg.s[i] * sg.s[j] * u);
+        }
+}
+
+// One thread per (p, k, g): abs-max of the group, scale, codes.
+__global__ void filter_quantize_kernel(const float *__restrict__ w32, int8_t *__restrict__ Wq,
+                                       float *__restrict__ sW, int P, int K, int C, int gs)
+{
+    const int G = C / gs;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)P * K * G) return;
+    const int g = (int)(idx % G);
+    const int k = (int)((idx / G) % K);
+    const int p = (int)(idx / ((long long)G * K));
+    const float *src = w32 + ((size_t)p * K + k) * C + (size_t)g * gs;
+    int8_t *dst = Wq + ((size_t)p * K + k) * C + (size_t)g * gs;
+    float amax = 0.f;
+    for (int e = 0; e < gs; ++e) amax = fmaxf(amax, fabsf(src[e]));
+    float scale = 0.f, inv = 0.f;
+    if (amax >= 1e-30f) {
+        scale = __fdiv_rn(amax, 127.f);
+        inv = __fdiv_rn(127.f, amax);
+    }
+    sW[((size_t)p * G + g) * K + k] = scale;
+    for (int e = 0; e < gs; ++e) {
+        int q = __float2int_rn(__fmul_rn(src[e], inv));
+        q = max(-127, min(127, q));
+        dst[e] = (int8_t)q;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *scratch_w32,
+                               cudaStream_t stream)
+{
+    const Geometry &g = plan.geo;
+    GScales sg;
+    for (int i = 0; i < kMaxN; ++i) sg.s[i] = i < g.n ? plan.sG[i] : 0.0;
+    {
+        const long long total = (long long)g.K * g.C;
+        const int threads = 128;
+        const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+        filter_transform_kernel<<<blocks, threads, 0, stream>>>(w_dev, scratch_w32, g.K, g.C, g.m, sg);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    {
+        const long long total = (long long)g.P * g.K * g.G;
+        const int threads = 128;
+        const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+        filter_quantize_kernel<<<blocks, threads, 0, stream>>>(scratch_w32, plan.Wq, plan.sW, g.P,
+                                                               g.K, g.C, g.gs);
+        return cudaGetLastError();
+    }
+}
+
+}  // namespace wfq

@@ -1,0 +1,91 @@
+// Internal declarations shared by the translation units of libwfq.so.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "wfq.h"
+
+namespace wfq {
+
+constexpr int kMaxN = 8;          // n = m + 2 <= 8
+constexpr int kMaxP = kMaxN * kMaxN;
+
+// Identifiers stored in the device status word when a bounded wait expires.
+enum WaitId : int {
+    kWaitSmemEmpty = 1,   // TMA producer waiting for a free pipeline stage
+    kWaitSmemFull = 2,    // MMA issuer waiting for TMA data
+    kWaitTmemEmpty = 3,   // MMA issuer waiting for a drained accumulator
+    kWaitTmemFull = 4,    // epilogue waiting for a finished accumulator
+    kWaitDrain = 5        // teardown waiting for copies in flight
+};
+
+// Geometry and scale tables handed to the kernels by value.
+struct Geometry {
+    int N, C, K, H, W;
+    int m, n, P;          // output tile, input tile, positions
+    int TH, TW, T, Tp;    // tiles per column/row, total, T rounded up to 32
+    int gs, G;            // channels per group, groups
+};
+
+// Per-position scale products, filled by the host in fp64 and rounded once.
+struct ScaleTables {
+    float in_scale[kMaxP];   // (sB_i/sBstd_i)*(sB_j/sBstd_j): applied after the
+                             // standard-scaled integer/rational input transform
+    float out_scale[kMaxP];  // sA_i*sA_j: applied before the output transform
+};
+
+struct Workspace {
+    int8_t *Xq = nullptr;   // [P][T][C]
+    float *sX = nullptr;    // [P][G][T]
+    float *Y = nullptr;     // [P][K][Tp]
+    size_t xq_bytes = 0, sx_bytes = 0, y_bytes = 0, total = 0;
+};
+
+}  // namespace wfq
+
+struct wfq_plan {
+    wfq::Geometry geo;
+    wfq_dtype_t in_dtype = WFQ_F32;
+    wfq::Workspace ws;
+    bool has_workspace = false;
+    bool prepared = false;
+    int device = -1;
+    int sm_count = 0;
+
+    // plan-owned device memory
+    int8_t *Wq = nullptr;      // [P][K][C]
+    float *sW = nullptr;       // [P][G][K]
+    int *status = nullptr;     // int32[4]
+    void *x_stage = nullptr;   // staging for wfq_conv_forward_host
+    float *y_stage = nullptr;
+
+    double sB[wfq::kMaxN], sG[wfq::kMaxN], sA[wfq::kMaxN];
+    wfq::ScaleTables tables;
+
+    CUtensorMap tmap_xq;       // Xq as (C, T, P) bytes, 128B-swizzled boxes
+    CUtensorMap tmap_wq;       // Wq as (C, K, P)
+    bool tmap_xq_ok = false, tmap_wq_ok = false;
+};
+
+namespace wfq {
+
+// Kernel launchers (one per translation unit).  Each returns a cudaError_t from the
+// launch; none synchronises.
+cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *scratch_w32,
+                               cudaStream_t stream);
+cudaError_t launch_input_transform(const wfq_plan &plan, const void *x_dev, cudaStream_t stream);
+cudaError_t launch_gemm(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t stream);
+cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStream_t stream);
+
+// Builds a 3-D byte tensor map (inner extent `inner`, rows, planes) with a
+// (128, box_rows, 1) box and 128-byte swizzle.  Returns false on failure.
+bool encode_tmap_bytes3d(CUtensorMap *map, const void *base, int inner, int rows, int planes,
+                         int box_rows);
+
+int gemm_block_n();   // output channels per CTA tile of the contraction kernel
+int gemm_block_m();   // tiles per CTA tile (128)
+
+}  // namespace wfq

@@ -1,0 +1,56 @@
+"""Full-size parity on sampled outputs: every layer of the benchmark configurations is
+run at its real size, in the launch configuration the benchmark times, and compared
+with the oracle on sampled tiles (the oracle evaluates the pipeline for a list of tiles;
+group scales are per tile and per output channel, so a tile's result does not depend
+on the other tiles).  Properties that hold at any size are checked on the whole output."""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2412_19867_b200 import binding as b
+from paper_2412_19867_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+FULL = ([L for L in wl.config_layers(2)] + [wl.config_layers(3)[i] for i in (0, 5, 8, 9)]
+        + wl.config_layers(4) + [wl.config_layers(5)[i] for i in (0, 1, 3, 5, 8)])
+
+
+@pytest.mark.parametrize("layer", FULL, ids=lambda L: L.name)
+def test_full_size_sampled_tiles(layer):
+    import torch
+    from tests.gpu_util import make_conv, codes_close, scales_close, max_rel, FINAL_TOL
+    conv, (x, w, sB, sG) = make_conv(layer)
+    xd = torch.from_numpy(x).cuda()
+    y = conv.forward(xd)
+    torch.cuda.synchronize()
+    conv.check_status()
+    yh = y.cpu().numpy()
+    assert np.isfinite(yh).all()
+
+    rng = np.random.default_rng(layer.seed)
+    T = conv.T
+    nt = min(T, 24)
+    tiles = np.unique(np.concatenate([[0, T - 1], rng.integers(0, T, nt)]))
+    ks = np.unique(np.concatenate([[0, layer.K - 1], rng.integers(0, layer.K, 46)]))
+    ref = orc.wfq(x, w[ks], layer.m, layer.gs, sB=sB, sG=sG, tiles=tiles)
+
+    Xq = conv.buffer(b.WFQ_BUF_XQ)[:, torch.from_numpy(tiles).cuda()].cpu().numpy()
+    codes_close(Xq, ref.Xq)
+    sX = conv.buffer(b.WFQ_BUF_SX)[:, :, torch.from_numpy(tiles).cuda()].cpu().numpy()
+    scales_close(sX, ref.sX.transpose(0, 2, 1))
+    Wq = conv.buffer(b.WFQ_BUF_WQ)[:, torch.from_numpy(ks).cuda()].cpu().numpy()
+    codes_close(Wq, ref.Wq)
+
+    m = layer.m
+    geo = orc.geometry(layer.N, layer.H, layer.W, m)
+    scale = np.max(np.abs(yh))
+    worst = 0.0
+    for i, t in enumerate(tiles):
+        tw, th, img = t % geo.TW, (t // geo.TW) % geo.TH, t // (geo.TW * geo.TH)
+        hh, ww = min(m, layer.H - th * m), min(m, layer.W - tw * m)
+        got = yh[img][ks][:, th * m:th * m + hh, tw * m:tw * m + ww]
+        want = ref.ytile[i][:, :hh, :ww]
+        worst = max(worst, float(np.max(np.abs(got - want))) / scale)
+    assert worst <= FINAL_TOL, worst
+    conv.close()
