@@ -45,6 +45,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=2, help="workload configuration 1..5")
     ap.add_argument("--impl", default="wfq", choices=["wfq", "reference"])
+    ap.add_argument("--only-layer", type=int, default=None,
+                    help="restrict the workload to one layer of the configuration (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=16.0,
@@ -59,6 +61,11 @@ def workload_name(cfg):
             3: "cfg3: ResNet-34-style sweep, N=64, 12 runs F(4,3)/F(6,3) x groups 32/64/128",
             4: "cfg4: diffusion-UNet block, N=2, C=K=320/640/1280 at 64/32/16, F(4,3), group 64",
             5: "cfg5: UNet conv-layer set at 128/64/32 latent, N=1, F(4,3) and F(6,3)"}[cfg]
+
+
+def select_layers(wl, args):
+    layers = wl.config_layers(args.config)
+    return layers if args.only_layer is None else [layers[args.only_layer]]
 
 
 # ---- byte counts the method itself must move (per launch) ----------------------------
@@ -176,7 +183,7 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from paper_2412_19867_b200 import workloads as wl
-    layers = wl.config_layers(args.config)
+    layers = select_layers(wl, args)
     tensors = [wl.make_tensors(L) for L in layers]
     nsteps = args.steps + args.warmup
     per_step = max(0.5, min(20.0, 90.0 / max(nsteps, 1)))
@@ -228,7 +235,7 @@ def run_wfq(args):
     torch.cuda.set_device(dev)
     stream = torch.cuda.current_stream(dev)
 
-    layers = wl.config_layers(args.config)
+    layers = select_layers(wl, args)
     tensors = [wl.make_tensors(L) for L in layers]
     convs, xs, ys = [], [], []
     for L, (x, w, sB, sG) in zip(layers, tensors):
@@ -364,7 +371,9 @@ def run_wfq(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-                "config": {"workload": workload_name(args.config), "layers": len(layers),
+                "config": {"workload": workload_name(args.config) +
+                           ("" if args.only_layer is None else f" (layer {args.only_layer} only)"),
+                           "layers": len(layers),
                            "l2": "flushed before every step (256 MiB memset outside the step's "
                                  "event pair)",
                            "parallelism": "replicas" if world > 1 else "single GPU"},
