@@ -57,7 +57,8 @@ typedef enum {
     WFQ_ERR_ALLOC = 3,        /* host or device allocation failed */
     WFQ_ERR_NOT_PREPARED = 4, /* workspace or filters missing */
     WFQ_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed */
-    WFQ_ERR_TIMEOUT = 6       /* a bounded device-side wait expired (status word) */
+    WFQ_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired (status word) */
+    WFQ_ERR_SCRATCH_TOO_SMALL = 7 /* problem larger than the library's built-in scratch */
 } wfq_status_t;
 
 typedef enum { WFQ_F32 = 0, WFQ_F16 = 1 } wfq_dtype_t;
@@ -118,6 +119,43 @@ wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t byte
  */
 wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const float *sB_host,
                                  const float *sG_host, const float *sA_host, void *stream);
+
+/*
+ * Filter quantization for callers that must not allocate.  (The paper has no
+ * counterpart to this call; it exists for integration reasons only.)
+ *
+ * wfq_prepare_filters obtains its buffers with cudaMalloc.  Some hosts of this library
+ * cannot do that at the point where filters arrive: code running inside a framework
+ * whose memory pool owns the whole device, a real-time loop where the allocator's
+ * implicit device synchronisation is not acceptable, or a process whose device memory
+ * was fully budgeted at start-up.  This call produces the same codes and scales as
+ * wfq_prepare_filters (same kernels, same arithmetic) and allocates nothing: no
+ * cudaMalloc/cudaFree, no host allocation, no library routine that allocates.  The fp32
+ * transformed filters it needs between its two kernels are kept in one array that is
+ * part of the library's device image, WFQ_STATIC_SCRATCH_FLOATS floats (16 MiB); every
+ * GPU on which the library is loaded holds that array until the process exits.
+ *
+ *   w_dev        device, fp32 [K][C][3][3]                               (input)
+ *   sG_host      host, m+2 floats, diagonal of S_G; NULL = standard scales
+ *   wq_dev       device, int8 [P][K][C], caller-owned                    (output)
+ *   sw_dev       device, fp32 [P][C/group_size][K], caller-owned         (output)
+ *   m in {4,6}; group_size a multiple of 32, at most 256, dividing C.
+ *
+ * Limit: (m+2)^2 * K * C <= WFQ_STATIC_SCRATCH_FLOATS, otherwise
+ * WFQ_ERR_SCRATCH_TOO_SMALL is returned and nothing is launched.  Other argument errors
+ * are reported as in wfq_prepare_filters.  Asynchronous on `stream`.
+ *
+ * The first call on each device looks up the device address of the built-in array
+ * (with that device current); make that first call outside any stream capture.  All
+ * calls on a device share the one array: it still holds the previous call's values
+ * when a call starts (harmless, every element that is read is written first by the
+ * same call, so nothing needs clearing), and two calls whose kernels can overlap on
+ * the GPU (different streams, or different host threads) race on it.  Serialise them.
+ */
+#define WFQ_STATIC_SCRATCH_FLOATS (4u * 1024u * 1024u)
+wfq_status_t wfq_quantize_filters_static(const float *w_dev, int K, int C, int m, int group_size,
+                                         const float *sG_host, int8_t *wq_dev, float *sw_dev,
+                                         void *stream);
 
 /*
  * The hot path: input transform + group quantization, per-position int8 tensor-core

@@ -12,7 +12,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwfq.so")
 
 WFQ_OK, WFQ_ERR_INVALID_ARG, WFQ_ERR_UNSUPPORTED, WFQ_ERR_ALLOC = 0, 1, 2, 3
-WFQ_ERR_NOT_PREPARED, WFQ_ERR_CUDA, WFQ_ERR_TIMEOUT = 4, 5, 6
+WFQ_ERR_NOT_PREPARED, WFQ_ERR_CUDA, WFQ_ERR_TIMEOUT, WFQ_ERR_SCRATCH_TOO_SMALL = 4, 5, 6, 7
+WFQ_STATIC_SCRATCH_FLOATS = 4 * 1024 * 1024
 WFQ_F32, WFQ_F16 = 0, 1
 WFQ_BUF_XQ, WFQ_BUF_SX, WFQ_BUF_WQ, WFQ_BUF_SW, WFQ_BUF_Y, WFQ_BUF_STATUS = range(6)
 
@@ -23,6 +24,7 @@ EXPORTS = [
     "wfq_conv_forward_host", "wfq_input_transform_quantize", "wfq_gemm_dequantize",
     "wfq_output_transform", "wfq_debug_gemm_acc32", "wfq_debug_get",
     "wfq_check_device_status", "wfq_plan_destroy", "wfq_status_string", "wfq_version",
+    "wfq_quantize_filters_static",
 ]
 
 _lib = None
@@ -59,6 +61,7 @@ def load():
     lib.wfq_debug_get.argtypes = [vp, ci, ctypes.POINTER(vp), ctypes.POINTER(sz)]
     lib.wfq_check_device_status.argtypes = [vp, vp, ctypes.POINTER(ci)]
     lib.wfq_plan_destroy.argtypes = [vp]
+    lib.wfq_quantize_filters_static.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
     lib.wfq_status_string.argtypes = [ci]
     lib.wfq_status_string.restype = ctypes.c_char_p
     lib.wfq_version.restype = ci
@@ -148,6 +151,13 @@ def wfq_check_device_status(plan, stream=0):
     where = ctypes.c_int(0)
     st = load().wfq_check_device_status(plan, stream, ctypes.byref(where))
     return st, where.value
+
+
+def wfq_quantize_filters_static(w_dev, K, C, m, group_size, sG, wq_dev, sw_dev, stream=0):
+    """Allocation-free filter quantization into caller-owned device buffers."""
+    keep, pg = _host_floats(sG)
+    _check(load().wfq_quantize_filters_static(w_dev, K, C, m, group_size, pg, wq_dev, sw_dev, stream),
+           "wfq_quantize_filters_static")
 
 
 def wfq_plan_destroy(plan):

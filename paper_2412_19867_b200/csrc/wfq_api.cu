@@ -84,6 +84,8 @@ const char *wfq_status_string(wfq_status_t s)
         case WFQ_ERR_NOT_PREPARED: return "plan has no workspace or no prepared filters";
         case WFQ_ERR_CUDA: return "CUDA call failed";
         case WFQ_ERR_TIMEOUT: return "device-side wait timed out";
+        case WFQ_ERR_SCRATCH_TOO_SMALL:
+            return "problem exceeds the library's built-in scratch array";
     }
     return "unknown status";
 }

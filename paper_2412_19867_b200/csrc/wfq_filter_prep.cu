@@ -1,6 +1,9 @@
 // Offline filter path: W = S_G V_G w V_G^T S_G (Section 4.1) in fp64, one rounding to
 // fp32, then group-wise int8 quantization along the input channels, stored
 // position-major Wq[P][K][C] with scales sW[P][G][K].  Not on the timed path.
+#include <cmath>
+#include <mutex>
+
 #include "wfq_internal.h"
 
 namespace wfq {
@@ -109,3 +112,88 @@ cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *
 }
 
 }  // namespace wfq
+
+// ---- filter quantization without any allocation -----------------------------------
+//
+// The fp32 transformed filters that sit between the two kernels above normally live in
+// a temporary device buffer.  Here they live in one fixed array inside the library's
+// device image, so the whole call needs no allocator at all.
+namespace wfq {
+namespace {
+
+constexpr size_t kStaticScratchFloats = WFQ_STATIC_SCRATCH_FLOATS;
+static __device__ __align__(256) float g_static_w32[kStaticScratchFloats];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+float *g_scratch_ptr[kMaxDevices];   // device address of g_static_w32, per device ordinal
+
+// `g_static_w32` is only a host-side handle in host code; the address a kernel can use
+// has to be asked for, with the device it is meant for current.
+cudaError_t static_scratch_address(int device, float **out)
+{
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[device]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_w32);
+        if (e != cudaSuccess) return e;
+        g_scratch_ptr[device] = static_cast<float *>(p);
+    }
+    *out = g_scratch_ptr[device];
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace wfq
+
+extern "C" wfq_status_t wfq_quantize_filters_static(const float *w_dev, int K, int C, int m,
+                                                    int group_size, const float *sG_host,
+                                                    int8_t *wq_dev, float *sw_dev, void *stream)
+{
+    using namespace wfq;
+    if (!w_dev || !wq_dev || !sw_dev) return WFQ_ERR_INVALID_ARG;
+    if (K < 1 || C < 1 || m < 1 || group_size < 1) return WFQ_ERR_INVALID_ARG;
+    if ((m != 4 && m != 6) || group_size % 32 != 0 || group_size > 256 || C % group_size != 0)
+        return WFQ_ERR_UNSUPPORTED;
+    const int n = m + 2, P = n * n;
+    const unsigned long long need = (unsigned long long)P * (unsigned long long)K * (unsigned long long)C;
+    if (need > kStaticScratchFloats) return WFQ_ERR_SCRATCH_TOO_SMALL;
+
+    static const double std4[6] = {1.0 / 4, -1.0 / 6, -1.0 / 6, 1.0 / 24, 1.0 / 24, 1.0};
+    static const double std6[8] = {1.0, -2.0 / 9, -2.0 / 9, 1.0 / 90, 1.0 / 90, 32.0 / 45, 32.0 / 45, 1.0};
+    GScales sg;
+    for (int i = 0; i < kMaxN; ++i) {
+        double v = 0.0;
+        if (i < n) {
+            v = sG_host ? (double)sG_host[i] : (m == 4 ? std4[i] : std6[i]);
+            if (!std::isfinite(v) || v == 0.0) return WFQ_ERR_INVALID_ARG;
+        }
+        sg.s[i] = v;
+    }
+
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return WFQ_ERR_CUDA;
+    if (device < 0 || device >= kMaxDevices) return WFQ_ERR_UNSUPPORTED;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess)
+        return WFQ_ERR_CUDA;
+    if (major != 10) return WFQ_ERR_UNSUPPORTED;
+    float *w32 = nullptr;
+    if (static_scratch_address(device, &w32) != cudaSuccess || !w32) return WFQ_ERR_CUDA;
+
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int threads = 128;
+    {
+        const long long total = (long long)K * C;
+        const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+        filter_transform_kernel<<<blocks, threads, 0, st>>>(w_dev, w32, K, C, m, sg);
+        if (cudaGetLastError() != cudaSuccess) return WFQ_ERR_CUDA;
+    }
+    {
+        const long long total = (long long)P * K * (C / group_size);
+        const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+        filter_quantize_kernel<<<blocks, threads, 0, st>>>(w32, wq_dev, sw_dev, P, K, C, group_size);
+        if (cudaGetLastError() != cudaSuccess) return WFQ_ERR_CUDA;
+    }
+    return WFQ_OK;
+}
