@@ -1,18 +1,24 @@
 // Fused input transform + group-wise int8 quantization.
 //
-//   X = S_B V_B x V_B^T S_B   (Section 4.1), fp32, never stored
+//   X = S_B V_B x V_B^T S_B   (Section 4.1), fp32, never stored to global memory
 //   per (position, tile, channel group): amax -> scale, codes (Section 2 quantizer,
 //   one scale per group, dynamic abs-max)
 //
-// A CTA stages a strip of the NCHW input (n rows x a chunk of tile columns x CB
-// channels, zero halo) in shared memory with coalesced row loads.  Work is then
-// handed out per (tile, channel group): L lanes cooperate on one group, each lane
-// owning CPL consecutive channels (gs = CPL*L*NSB), so the codes of a lane pack into
-// one 8/16/32-bit store and the group abs-max is a warp-level reduction
-// (group_absmax: redux.sync over the whole warp, or a shuffle butterfly over L lanes).
-// The 2-D transform uses the standard-scaled matrix B^T (small integers / dyadic
-// rationals, hard-coded as add/fma chains); the caller's scales enter as one
-// per-position factor.
+// One CTA handles TB neighbouring tiles of one tile row and CB input channels (one or
+// two whole groups).  Three steps, separated by block barriers:
+//   stage    the zero-padded input strip (n rows x 16 columns x CB channels) goes to
+//            shared memory with 4-byte cp.async copies, all in flight at once
+//   phase 1  thread <-> (tile, channel): the n x n patch is transformed with the
+//            standard-scaled B^T (small integers / dyadic rationals as add/fma chains),
+//            multiplied by the caller's per-position factor and written as fp32 to a
+//            shared [tile][channel][position] array (odd pitch: conflict free)
+//   phase 2  thread <-> (tile, group, position): it reads the group's values of that
+//            position (lanes along the position: conflict free), takes the abs-max
+//            serially, derives scale and reciprocal once, rounds with the 1.5*2^23
+//            trick (same result as mul + round-half-even convert) and stores 16 codes
+//            per 16-byte store.
+// The abs-max over a group therefore needs no shuffles; for groups of more than 64
+// channels phase 2 reads shared memory twice instead of holding the group in registers.
 #include <cuda_fp16.h>
 
 #include "wfq_internal.h"
@@ -20,13 +26,16 @@
 namespace wfq {
 namespace {
 
+constexpr int K1_THREADS = 128;
+constexpr int K1_WP = 16;        // staged columns per row (image columns w_base .. w_base+15)
+
 struct K1Params {
-    int TWC;      // tiles per column chunk
-    int NCH;      // chunks per strip
-    int CB;       // channels per CTA
-    int Wp;       // smem row pitch (elements)
-    int CS;       // smem channel stride (elements)
-    int NSB;      // channel sub-blocks per group (gs = CPL*L*NSB)
+    int TB;            // tiles per CTA
+    int NCH;           // chunks of TB tiles per tile row
+    int CB;            // channels per CTA (a multiple of the group size)
+    int CS;            // shared-memory channel stride of the strip (elements)
+    int strip_bytes;   // bytes of the strip, rounded up to 16
+    int pair;          // 1: rows can be copied as aligned element pairs
 };
 
 // ---- 1-D input transforms with the standard B^T ------------------------------------
@@ -68,29 +77,16 @@ __device__ __forceinline__ void bt_1d(const float (&d)[8], float (&r)[8])
     r[6] = f - g;
 }
 
-// ---- group abs-max over L lanes (L a power of two, lanes of a group adjacent) -------
-template <int L>
-__device__ __forceinline__ float group_absmax(float v)   // v >= 0
-{
-    if constexpr (L == 32) {
-        // non-negative floats order like their bit patterns
-        return __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(v)));
-    } else {
-#pragma unroll
-        for (int o = L / 2; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-        return v;
-    }
-}
 
 // ---- patch load from the staged strip ---------------------------------------------
 // `ch` points at the channel's plane in smem; `col0` is the (even) smem column whose
 // successor is the tile's first input column.
 template <int NN>
-__device__ __forceinline__ void load_patch(const __half *ch, int col0, int Wp, float (&d)[NN][NN])
+__device__ __forceinline__ void load_patch(const __half *ch, int col0, float (&d)[NN][NN])
 {
 #pragma unroll
     for (int a = 0; a < NN; ++a) {
-        const __half2 *row = reinterpret_cast<const __half2 *>(ch + a * Wp + col0);
+        const __half2 *row = reinterpret_cast<const __half2 *>(ch + a * K1_WP + col0);
         float v[NN + 2];
 #pragma unroll
         for (int w = 0; w < (NN + 2) / 2; ++w) {
@@ -104,18 +100,96 @@ __device__ __forceinline__ void load_patch(const __half *ch, int col0, int Wp, f
 }
 
 template <int NN>
-__device__ __forceinline__ void load_patch(const float *ch, int col0, int Wp, float (&d)[NN][NN])
+__device__ __forceinline__ void load_patch(const float *ch, int col0, float (&d)[NN][NN])
 {
 #pragma unroll
     for (int a = 0; a < NN; ++a)
 #pragma unroll
-        for (int b = 0; b < NN; ++b) d[a][b] = ch[a * Wp + col0 + 1 + b];
+        for (int b = 0; b < NN; ++b) d[a][b] = ch[a * K1_WP + col0 + 1 + b];
 }
 
-// Z = B^T d B with the standard B^T, then the caller's per-position factor.
+// Round v*inv to the nearest integer (ties to even) and return it in the low byte:
+// fl32(v*inv) + 1.5*2^23 is exact up to the rounding to an integer, and the sum's
+// bit pattern is 0x4B400000 + q for |q| <= 2^22.
+__device__ __forceinline__ uint32_t code_bits(float v, float inv)
+{
+    return __float_as_uint(__fadd_rn(__fmul_rn(v, inv), 12582912.f));
+}
+
+__device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
+
+__device__ __forceinline__ void cp_async_4(uint32_t dst, const void *src, bool valid)
+{
+    const int n = valid ? 4 : 0;   // 0 source bytes: the destination is zero filled
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
+// ---- strip staging -----------------------------------------------------------------
+// smem column j of the strip holds image column w_base + j (w_base even); rows are
+// image rows h_base .. h_base + NN - 1; anything outside the image is zero.
+template <typename Tin, int NN>
+__device__ __forceinline__ void stage_strip(Tin *sm, const Tin *__restrict__ x, const Geometry &g,
+                                            const K1Params &prm, int img, int c_base, int h_base,
+                                            int w_base)
+{
+    const size_t HW = (size_t)g.H * g.W;
+    const Tin *ximg = x + ((size_t)img * g.C + c_base) * HW;
+    if (sizeof(Tin) == 4) {
+        // fp32: one 4-byte copy per element (the odd channel stride rules out 8-byte ones)
+        const int total = prm.CB * NN * K1_WP;
+        const uint32_t sm_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(sm));
+        for (int idx = threadIdx.x; idx < total; idx += K1_THREADS) {
+            const int j = idx % K1_WP;
+            const int row = idx / K1_WP;
+            const int c = row / NN, a = row - c * NN;
+            const int h = h_base + a, w = w_base + j;
+            const bool ok = h >= 0 && h < g.H && w >= 0 && w < g.W;
+            const Tin *src = ok ? ximg + (size_t)c * HW + (size_t)h * g.W + w : x;
+            cp_async_4(sm_u32 + (uint32_t)((c * prm.CS + a * K1_WP + j) * 4), src, ok);
+        }
+        cp_async_wait_all();
+    } else if (prm.pair) {
+        // fp16, even W, 4-byte aligned base: one 4-byte copy per pair of columns
+        constexpr int PR = K1_WP / 2;
+        const int total = prm.CB * NN * PR;
+        const uint32_t sm_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(sm));
+        for (int idx = threadIdx.x; idx < total; idx += K1_THREADS) {
+            const int jp = idx % PR;
+            const int row = idx / PR;
+            const int c = row / NN, a = row - c * NN;
+            const int h = h_base + a, w = w_base + 2 * jp;
+            const bool ok = h >= 0 && h < g.H && w >= 0 && w < g.W;   // W even: both or none
+            const Tin *src = ok ? ximg + (size_t)c * HW + (size_t)h * g.W + w : x;
+            cp_async_4(sm_u32 + (uint32_t)((c * prm.CS + a * K1_WP + 2 * jp) * 2), src, ok);
+        }
+        cp_async_wait_all();
+    } else {
+        const int total = prm.CB * NN * K1_WP;
+        for (int idx = threadIdx.x; idx < total; idx += K1_THREADS) {
+            const int j = idx % K1_WP;
+            const int row = idx / K1_WP;
+            const int c = row / NN, a = row - c * NN;
+            const int h = h_base + a, w = w_base + j;
+            Tin v = Tin(0);
+            if (h >= 0 && h < g.H && w >= 0 && w < g.W)
+                v = __ldg(ximg + (size_t)c * HW + (size_t)h * g.W + w);
+            sm[c * prm.CS + a * K1_WP + j] = v;
+        }
+    }
+}
+
+// Z = B^T d B with the standard B^T, times the caller's per-position factor, written
+// to out[p] for p = i*NN + j.
 template <int NN>
 __device__ __forceinline__ void transform_patch(float (&d)[NN][NN], const ScaleTables &tab,
-                                                float (&X)[NN * NN])
+                                                float *__restrict__ out)
 {
 #pragma unroll
     for (int b = 0; b < NN; ++b) {   // columns: d <- B^T d
@@ -131,222 +205,140 @@ __device__ __forceinline__ void transform_patch(float (&d)[NN][NN], const ScaleT
         float r[NN];
         bt_1d(d[i], r);
 #pragma unroll
-        for (int j = 0; j < NN; ++j) X[i * NN + j] = __fmul_rn(r[j], tab.in_scale[i * NN + j]);
+        for (int j = 0; j < NN; ++j) out[i * NN + j] = __fmul_rn(r[j], tab.in_scale[i * NN + j]);
     }
 }
 
-__device__ __forceinline__ int quantize_code(float v, float inv)
+// ---- group abs-max and scale (the quantizer of Section 2, one scale per group) ------
+// amax >= 0.  Returns the stored scale and the reciprocal used for the codes.
+__device__ __forceinline__ void group_scale(float amax, float &scale, float &inv)
 {
-    const int q = __float2int_rn(__fmul_rn(v, inv));   // round half to even
-    return max(-127, min(127, q));
-}
-
-template <int CPL>
-__device__ __forceinline__ void store_codes(int8_t *dst, const int (&q)[CPL])
-{
-    if constexpr (CPL == 4) {
-        const uint32_t w = (uint32_t)(q[0] & 0xff) | ((uint32_t)(q[1] & 0xff) << 8) |
-                           ((uint32_t)(q[2] & 0xff) << 16) | ((uint32_t)(q[3] & 0xff) << 24);
-        *reinterpret_cast<uint32_t *>(dst) = w;
-    } else if constexpr (CPL == 2) {
-        *reinterpret_cast<uint16_t *>(dst) = (uint16_t)((q[0] & 0xff) | ((q[1] & 0xff) << 8));
-    } else {
-        dst[0] = (int8_t)q[0];
-    }
-}
-
-// ---- strip staging -----------------------------------------------------------------
-// smem column j of the strip holds image column w_base + j (w_base even); rows are
-// image rows h_base .. h_base + NN - 1; anything outside the image is zero.
-template <typename Tin>
-__device__ __forceinline__ void stage_strip(Tin *sm, const Tin *__restrict__ x, const Geometry &g,
-                                            const K1Params &prm, int NN, int img, int c_base,
-                                            int h_base, int w_base, int cols)
-{
-    const size_t HW = (size_t)g.H * g.W;
-    const Tin *ximg = x + (size_t)img * g.C * HW;
-    if ((g.W & 1) == 0 && sizeof(Tin) == 2) {
-        // pairs of halves: 4-byte global loads and shared stores
-        const int pairs = cols / 2;
-        const int total = prm.CB * NN * pairs;
-        for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
-            const int jp = idx % pairs;
-            const int a = (idx / pairs) % NN;
-            const int c = idx / (pairs * NN);
-            const int h = h_base + a, w = w_base + 2 * jp;
-            uint32_t v = 0u;
-            if (h >= 0 && h < g.H && w >= 0 && w < g.W)
-                v = __ldg(reinterpret_cast<const uint32_t *>(ximg + (size_t)(c_base + c) * HW +
-                                                             (size_t)h * g.W + w));
-            *reinterpret_cast<uint32_t *>(sm + (size_t)c * prm.CS + a * prm.Wp + 2 * jp) = v;
-        }
-    } else {
-        const int total = prm.CB * NN * cols;
-        for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
-            const int j = idx % cols;
-            const int a = (idx / cols) % NN;
-            const int c = idx / (cols * NN);
-            const int h = h_base + a, w = w_base + j;
-            Tin v = Tin(0);
-            if (h >= 0 && h < g.H && w >= 0 && w < g.W)
-                v = __ldg(ximg + (size_t)(c_base + c) * HW + (size_t)h * g.W + w);
-            sm[(size_t)c * prm.CS + a * prm.Wp + j] = v;
-        }
-    }
+    const bool nz = amax >= 1e-30f;
+    scale = nz ? __fdiv_rn(amax, 127.f) : 0.f;
+    inv = nz ? __fdiv_rn(127.f, amax) : 0.f;
 }
 
 // ---- the kernel ----------------------------------------------------------------------
-template <int M, typename Tin, int CPL, int L>
-__global__ void __launch_bounds__(256)
+// GSR > 0: compile-time group size held in registers during phase 2 (32 or 64);
+// GSR == 0: any group size, phase 2 reads shared memory twice.
+template <int M, typename Tin, int GSR>
+__global__ void __launch_bounds__(K1_THREADS, 4)
 input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
                        float *__restrict__ sX, Geometry g, ScaleTables tab, K1Params prm)
 {
     constexpr int NN = M + 2;
     constexpr int P = NN * NN;
-    constexpr int TPW = 32 / L;          // tiles per warp step
+    constexpr int PP = P + 1;                      // odd pitch of the [channel][position] array
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    Tin *sm = reinterpret_cast<Tin *>(smem_raw);
+    Tin *strip = reinterpret_cast<Tin *>(smem_raw);
+    float *Xs = reinterpret_cast<float *>(smem_raw + prm.strip_bytes);
 
-    const int strip = blockIdx.x / prm.NCH;       // img*TH + th
-    const int chunk = blockIdx.x % prm.NCH;
-    const int img = strip / g.TH, th = strip % g.TH;
-    const int tw0 = chunk * prm.TWC;
-    const int ntile = min(prm.TWC, g.TW - tw0);
+    const int srow = blockIdx.x / prm.NCH;         // img*TH + th
+    const int chunk = blockIdx.x - srow * prm.NCH;
+    const int img = srow / g.TH, th = srow - img * g.TH;
+    const int tw0 = chunk * prm.TB;
+    const int ntile = min(prm.TB, g.TW - tw0);
     const int c_base = blockIdx.y * prm.CB;
-    const int h_base = th * M - 1;
-    const int w_base = tw0 * M - 2;
-    const int cols = prm.Wp;                      // every staged column is initialised
 
-    stage_strip<Tin>(sm, x, g, prm, NN, img, c_base, h_base, w_base, cols);
+    stage_strip<Tin, NN>(strip, x, g, prm, img, c_base, th * M - 1, tw0 * M - 2);
     __syncthreads();
 
+    // ---- phase 1: transform, one (tile, channel) per thread --------------------------
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nwarps = blockDim.x >> 5;
-    const int q = lane % L, ti = lane / L;
-    const int groups = prm.CB / g.gs;
-    const int tblocks = (ntile + TPW - 1) / TPW;
-    const int items = tblocks * groups;
+    constexpr int NWARP = K1_THREADS / 32;
+    const int cb32 = prm.CB >> 5;
+    for (int wt = warp; wt < ntile * cb32; wt += NWARP) {
+        const int tl = wt / cb32;
+        const int c = (wt - tl * cb32) * 32 + lane;
+        float d[NN][NN];
+        load_patch<NN>(strip + c * prm.CS, tl * M, d);
+        transform_patch<NN>(d, tab, Xs + (size_t)(tl * prm.CB + c) * PP);
+    }
+    __syncthreads();
 
-    for (int it = warp; it < items; it += nwarps) {
-        const int grp = it % groups, tb = it / groups;
-        const int tl = tb * TPW + ti;             // tile within the chunk
-        const bool valid = tl < ntile;
-        const int tlc = valid ? tl : ntile - 1;   // clamp: idle lanes recompute a real tile
-        const int col0 = tlc * M;                 // smem column before the tile's first one
-        const int t = (strip * g.TW) + tw0 + tlc; // global tile id
-        const int gglob = c_base / g.gs + grp;
-        const int c_grp = grp * g.gs;             // first channel of the group within CB
-
-        float amax[P];
+    // ---- phase 2: quantize, one (tile, group, position) per thread -------------------
+    const int gs = GSR > 0 ? GSR : g.gs;
+    const int ng = prm.CB / gs;
+    const int g_base = c_base / gs;
+    const int tasks = ntile * ng * P;
+    for (int task = threadIdx.x; task < tasks; task += K1_THREADS) {
+        const int q = task / P, p = task - q * P;
+        const int tl = q / ng, grp = q - tl * ng;
+        const int t = srow * g.TW + tw0 + tl;
+        const float *src = Xs + (size_t)(tl * prm.CB + grp * gs) * PP + p;
+        int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
+        float scale, inv;
+        if constexpr (GSR > 0) {
+            float v[GSR];
+            float amax = 0.f;
 #pragma unroll
-        for (int p = 0; p < P; ++p) amax[p] = 0.f;
-
-        if (prm.NSB == 1) {
-            // single pass: transformed values stay in registers
-            float X[CPL][P];
-#pragma unroll
-            for (int j = 0; j < CPL; ++j) {
-                float d[NN][NN];
-                load_patch<NN>(sm + (size_t)(c_grp + q * CPL + j) * prm.CS, col0, prm.Wp, d);
-                transform_patch<NN>(d, tab, X[j]);
-#pragma unroll
-                for (int p = 0; p < P; ++p) amax[p] = fmaxf(amax[p], fabsf(X[j][p]));
+            for (int cc = 0; cc < GSR; ++cc) {
+                v[cc] = src[cc * PP];
+                amax = fmaxf(amax, fabsf(v[cc]));
             }
-            const int c_out = c_base + c_grp + q * CPL;
+            group_scale(amax, scale, inv);
 #pragma unroll
-            for (int p = 0; p < P; ++p) {
-                const float am = group_absmax<L>(amax[p]);
-                const bool nz = am >= 1e-30f;
-                const float scale = nz ? __fdiv_rn(am, 127.f) : 0.f;
-                const float inv = nz ? __fdiv_rn(127.f, am) : 0.f;
-                int code[CPL];
+            for (int c16 = 0; c16 < GSR; c16 += 16) {
+                uint32_t wd[4];
 #pragma unroll
-                for (int j = 0; j < CPL; ++j) code[j] = quantize_code(X[j][p], inv);
-                if (valid) {
-                    store_codes<CPL>(Xq + ((size_t)p * g.T + t) * g.C + c_out, code);
-                    if (q == 0) sX[((size_t)p * g.G + gglob) * g.T + t] = scale;
-                }
+                for (int k = 0; k < 4; ++k)
+                    wd[k] = pack4(code_bits(v[c16 + 4 * k], inv), code_bits(v[c16 + 4 * k + 1], inv),
+                                  code_bits(v[c16 + 4 * k + 2], inv), code_bits(v[c16 + 4 * k + 3], inv));
+                *reinterpret_cast<uint4 *>(dst + c16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
             }
         } else {
-            // two passes over the group's sub-blocks: maxima first, then recompute
-            for (int sb = 0; sb < prm.NSB; ++sb) {
+            float amax = 0.f;
+            for (int cc = 0; cc < gs; ++cc) amax = fmaxf(amax, fabsf(src[cc * PP]));
+            group_scale(amax, scale, inv);
+            for (int c16 = 0; c16 < gs; c16 += 16) {
+                uint32_t wd[4];
 #pragma unroll
-                for (int j = 0; j < CPL; ++j) {
-                    float d[NN][NN], X[P];
-                    const int cl = c_grp + (sb * L + q) * CPL + j;
-                    load_patch<NN>(sm + (size_t)cl * prm.CS, col0, prm.Wp, d);
-                    transform_patch<NN>(d, tab, X);
-#pragma unroll
-                    for (int p = 0; p < P; ++p) amax[p] = fmaxf(amax[p], fabsf(X[p]));
+                for (int k = 0; k < 4; ++k) {
+                    const float *s4 = src + (size_t)(c16 + 4 * k) * PP;
+                    wd[k] = pack4(code_bits(s4[0], inv), code_bits(s4[PP], inv),
+                                  code_bits(s4[2 * PP], inv), code_bits(s4[3 * PP], inv));
                 }
-            }
-#pragma unroll
-            for (int p = 0; p < P; ++p) {
-                const float am = group_absmax<L>(amax[p]);
-                const bool nz = am >= 1e-30f;
-                if (valid && q == 0)
-                    sX[((size_t)p * g.G + gglob) * g.T + t] = nz ? __fdiv_rn(am, 127.f) : 0.f;
-                amax[p] = nz ? __fdiv_rn(127.f, am) : 0.f;   // now holds inv
-            }
-            for (int sb = 0; sb < prm.NSB; ++sb) {
-                float X[CPL][P];
-#pragma unroll
-                for (int j = 0; j < CPL; ++j) {
-                    float d[NN][NN];
-                    const int cl = c_grp + (sb * L + q) * CPL + j;
-                    load_patch<NN>(sm + (size_t)cl * prm.CS, col0, prm.Wp, d);
-                    transform_patch<NN>(d, tab, X[j]);
-                }
-                const int c_out = c_base + c_grp + (sb * L + q) * CPL;
-#pragma unroll
-                for (int p = 0; p < P; ++p) {
-                    int code[CPL];
-#pragma unroll
-                    for (int j = 0; j < CPL; ++j) code[j] = quantize_code(X[j][p], amax[p]);
-                    if (valid) store_codes<CPL>(Xq + ((size_t)p * g.T + t) * g.C + c_out, code);
-                }
+                *reinterpret_cast<uint4 *>(dst + c16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
             }
         }
+        sX[((size_t)p * g.G + g_base + grp) * g.T + t] = scale;
     }
 }
 
-template <int M, typename Tin, int CPL, int L>
+template <int M, typename Tin, int GSR>
 cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stream)
 {
     const Geometry &g = plan.geo;
     constexpr int NN = M + 2;
-    K1Params prm;
-    prm.NSB = g.gs / (CPL * L);
-    prm.CB = g.gs;                         // one group per CTA row keeps the strip small
-    if (g.gs < 64 && g.C % 64 == 0) prm.CB = 64;
-    // tiles per chunk: a multiple of 4 (so chunk starts stay 16-byte friendly), sized
-    // so the strip stays below ~48 KB
+    constexpr int PP = NN * NN + 1;
     const int esz = (int)sizeof(Tin);
-    int twc = g.TW;
-    auto strip_bytes = [&](int tiles, int &Wp, int &CS) {
-        Wp = (tiles * M + 4 + 7) / 8 * 8;          // 2 left pad + tiles*M + 1 halo + slack
-        CS = NN * Wp;
-        // channel stride: an odd number of 32-bit words (bank-conflict-free lane stride)
-        if (esz == 2) { CS += 2; if ((CS / 2) % 2 == 0) CS += 2; }
-        else { if (CS % 2 == 0) CS += 1; }
-        return (size_t)prm.CB * CS * esz;
+    K1Params prm;
+    prm.TB = (K1_WP - 3) / M;                      // 2 tiles for F(6,3), 3 for F(4,3)
+    prm.CB = g.gs;
+    if (g.gs == 32 && g.C % 64 == 0) prm.CB = 64;  // two groups per CTA
+    // channel stride: an odd number of 32-bit words, so lanes that walk over channels
+    // hit different banks
+    int cs = NN * K1_WP;
+    if (esz == 2) { cs += 2; if ((cs / 2) % 2 == 0) cs += 2; }
+    else if (cs % 2 == 0) cs += 1;
+    prm.CS = cs;
+    prm.strip_bytes = (prm.CB * cs * esz + 15) / 16 * 16;
+    prm.pair = (g.W % 2 == 0) && (reinterpret_cast<uintptr_t>(x_dev) % 4 == 0);
+    auto smem_bytes = [&]() {
+        return (size_t)prm.strip_bytes + (size_t)prm.TB * prm.CB * PP * sizeof(float);
     };
-    int Wp = 0, CS = 0;
-    while (twc > 4 && strip_bytes(twc, Wp, CS) > 48 * 1024) twc = (twc / 2 + 3) / 4 * 4;
-    const size_t smem = strip_bytes(twc, Wp, CS);
-    prm.TWC = twc;
-    prm.NCH = (g.TW + twc - 1) / twc;
-    prm.Wp = Wp;
-    prm.CS = CS;
+    while (prm.TB > 1 && smem_bytes() > 220 * 1024) --prm.TB;   // very large groups
+    const size_t smem = smem_bytes();
+    prm.NCH = (g.TW + prm.TB - 1) / prm.TB;
 
-    auto kern = input_transform_kernel<M, Tin, CPL, L>;
+    auto kern = input_transform_kernel<M, Tin, GSR>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
     dim3 grid((unsigned)(g.N * g.TH * prm.NCH), (unsigned)(g.C / prm.CB));
-    kern<<<grid, 256, smem, stream>>>(static_cast<const Tin *>(x_dev), plan.ws.Xq, plan.ws.sX, g,
-                                      plan.tables, prm);
+    kern<<<grid, K1_THREADS, smem, stream>>>(static_cast<const Tin *>(x_dev), plan.ws.Xq, plan.ws.sX, g,
+                                             plan.tables, prm);
     return cudaGetLastError();
 }
 
@@ -354,16 +346,9 @@ template <int M, typename Tin>
 cudaError_t dispatch_gs(const wfq_plan &plan, const void *x, cudaStream_t s)
 {
     const int gs = plan.geo.gs;
-    if constexpr (M == 4) {
-        if (gs == 32) return launch_k1<4, Tin, 4, 8>(plan, x, s);
-        if (gs == 64) return launch_k1<4, Tin, 4, 16>(plan, x, s);
-        if (gs % 128 == 0) return launch_k1<4, Tin, 4, 32>(plan, x, s);
-        return launch_k1<4, Tin, 4, 8>(plan, x, s);      // 96, 160, 192, 224: sub-blocks of 32
-    } else {
-        if (gs == 32) return launch_k1<6, Tin, 2, 16>(plan, x, s);
-        if (gs % 64 == 0) return launch_k1<6, Tin, 2, 32>(plan, x, s);
-        return launch_k1<6, Tin, 2, 16>(plan, x, s);
-    }
+    if (gs == 32) return launch_k1<M, Tin, 32>(plan, x, s);
+    if (gs == 64) return launch_k1<M, Tin, 64>(plan, x, s);
+    return launch_k1<M, Tin, 0>(plan, x, s);
 }
 
 }  // namespace
