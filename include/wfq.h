@@ -66,9 +66,11 @@ typedef enum { WFQ_F32 = 0, WFQ_F16 = 1 } wfq_dtype_t;
 /* Buffers that wfq_debug_get can expose (all device memory). */
 typedef enum {
     WFQ_BUF_XQ = 0,     /* int8  Xq[P][T][C]            (workspace)  */
-    WFQ_BUF_SX = 1,     /* fp32  sX[P][G][T]            (workspace)  */
+    WFQ_BUF_SX = 1,     /* fp32  sX[P][G][Ts], Ts = T rounded up to 128; entries t >= T
+                           are not written (workspace)  */
     WFQ_BUF_WQ = 2,     /* int8  Wq[P][K][C]            (plan-owned) */
-    WFQ_BUF_SW = 3,     /* fp32  sW[P][G][K]            (plan-owned) */
+    WFQ_BUF_SW = 3,     /* fp32  sW[P][G][Kp], Kp = K rounded up to 128, zero for k >= K
+                           (plan-owned) */
     WFQ_BUF_Y = 4,      /* fp32  Y[P][K][Tp], Tp = T rounded up to 32 (workspace) */
     WFQ_BUF_STATUS = 5  /* int32 status[4]: {code, where, block, aux} (plan-owned) */
 } wfq_buffer_t;

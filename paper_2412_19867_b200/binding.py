@@ -197,6 +197,8 @@ class Conv:
         self.P, self.G = n * n, C // group_size
         self.T = N * (-(-H // m)) * (-(-W // m))
         self.Tp = (self.T + 31) // 32 * 32
+        self.Ts = (self.T + 127) // 128 * 128
+        self.Kp = (K + 127) // 128 * 128
 
     def _stream(self):
         return self.torch.cuda.current_stream(self.device).cuda_stream
@@ -230,9 +232,9 @@ class Conv:
         ptr, nbytes = wfq_debug_get(self.plan, which)
         N, C, K, H, W = self.shape
         shapes = {WFQ_BUF_XQ: ((self.P, self.T, C), "|i1", 1),
-                  WFQ_BUF_SX: ((self.P, self.G, self.T), "<f4", 4),
+                  WFQ_BUF_SX: ((self.P, self.G, self.Ts), "<f4", 4),
                   WFQ_BUF_WQ: ((self.P, K, C), "|i1", 1),
-                  WFQ_BUF_SW: ((self.P, self.G, K), "<f4", 4),
+                  WFQ_BUF_SW: ((self.P, self.G, self.Kp), "<f4", 4),
                   WFQ_BUF_Y: ((self.P, K, self.Tp), "<f4", 4),
                   WFQ_BUF_STATUS: ((4,), "<i4", 4)}
         shape, typestr, esz = shapes[which]

@@ -116,11 +116,13 @@ wfq_status_t wfq_plan_create(wfq_plan_t **out, int N, int C, int K, int H, int W
         return WFQ_ERR_UNSUPPORTED;
     }
     g.T = (int)T; g.Tp = (g.T + 31) / 32 * 32;
+    g.Ts = (g.T + 127) / 128 * 128; g.Kp = (K + 127) / 128 * 128;
     g.gs = group_size; g.G = C / group_size;
+    wfq::gemm_choose(g, &p->gemm_swap, &p->gemm_bn);
 
     wfq::Workspace &ws = p->ws;
     ws.xq_bytes = align_up((size_t)g.P * g.T * g.C, 1024);
-    ws.sx_bytes = align_up((size_t)g.P * g.G * g.T * sizeof(float), 1024);
+    ws.sx_bytes = align_up((size_t)g.P * g.G * g.Ts * sizeof(float), 1024);
     ws.y_bytes = align_up((size_t)g.P * g.K * g.Tp * sizeof(float), 1024);
     ws.total = ws.xq_bytes + ws.sx_bytes + ws.y_bytes;
     *out = p;
@@ -149,7 +151,7 @@ wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t byte
     ws.Y = reinterpret_cast<float *>(base + ws.xq_bytes + ws.sx_bytes);
     const wfq::Geometry &g = plan->geo;
     plan->tmap_xq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_xq, ws.Xq, g.C, g.T, g.P,
-                                               wfq::gemm_block_m());
+                                               plan->gemm_swap ? plan->gemm_bn : wfq::gemm_block_m());
     if (!plan->tmap_xq_ok) return WFQ_ERR_CUDA;
     plan->has_workspace = true;
     return WFQ_OK;
@@ -192,9 +194,14 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
     plan->sm_count = prop.multiProcessorCount;
 
     const size_t wq_bytes = (size_t)g.P * g.K * g.C;
-    const size_t sw_bytes = (size_t)g.P * g.G * g.K * sizeof(float);
+    const size_t sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
     if (!plan->Wq && (e = cudaMalloc(&plan->Wq, wq_bytes)) != cudaSuccess) return cuda_status(e);
-    if (!plan->sW && (e = cudaMalloc(&plan->sW, sw_bytes)) != cudaSuccess) return cuda_status(e);
+    if (!plan->sW) {
+        if ((e = cudaMalloc(&plan->sW, sw_bytes)) != cudaSuccess) return cuda_status(e);
+        // the padding columns k >= K stay zero
+        if ((e = cudaMemsetAsync(plan->sW, 0, sw_bytes, as_stream(stream))) != cudaSuccess)
+            return WFQ_ERR_CUDA;
+    }
     if (!plan->status) {
         if ((e = cudaMalloc(&plan->status, 4 * sizeof(int))) != cudaSuccess) return cuda_status(e);
         if ((e = cudaMemsetAsync(plan->status, 0, 4 * sizeof(int), as_stream(stream))) != cudaSuccess)
@@ -208,7 +215,7 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
     if (e != cudaSuccess || e2 != cudaSuccess) return WFQ_ERR_CUDA;
 
     plan->tmap_wq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_wq, plan->Wq, g.C, g.K, g.P,
-                                               wfq::gemm_block_n());
+                                               plan->gemm_swap ? wfq::gemm_block_m() : plan->gemm_bn);
     if (!plan->tmap_wq_ok) return WFQ_ERR_CUDA;
     plan->prepared = true;
     return WFQ_OK;
@@ -226,7 +233,7 @@ wfq_status_t wfq_gemm_dequantize(wfq_plan_t *plan, void *stream)
 {
     wfq_status_t s = ready_to_run(plan);
     if (s != WFQ_OK) return s;
-    return cuda_status(wfq::launch_gemm(*plan, nullptr, as_stream(stream)));
+    return cuda_status(wfq::launch_gemm(*plan, nullptr, as_stream(stream), false));
 }
 
 wfq_status_t wfq_debug_gemm_acc32(wfq_plan_t *plan, int32_t *acc_dev, void *stream)
@@ -234,7 +241,7 @@ wfq_status_t wfq_debug_gemm_acc32(wfq_plan_t *plan, int32_t *acc_dev, void *stre
     wfq_status_t s = ready_to_run(plan);
     if (s != WFQ_OK) return s;
     if (!acc_dev) return WFQ_ERR_INVALID_ARG;
-    return cuda_status(wfq::launch_gemm(*plan, acc_dev, as_stream(stream)));
+    return cuda_status(wfq::launch_gemm(*plan, acc_dev, as_stream(stream), false));
 }
 
 wfq_status_t wfq_output_transform(wfq_plan_t *plan, float *y_dev, void *stream)
@@ -242,7 +249,7 @@ wfq_status_t wfq_output_transform(wfq_plan_t *plan, float *y_dev, void *stream)
     wfq_status_t s = ready_to_run(plan);
     if (s != WFQ_OK) return s;
     if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 15u)) return WFQ_ERR_INVALID_ARG;
-    return cuda_status(wfq::launch_output_transform(*plan, y_dev, as_stream(stream)));
+    return cuda_status(wfq::launch_output_transform(*plan, y_dev, as_stream(stream), false));
 }
 
 wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev, void *stream)
@@ -254,8 +261,8 @@ wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev,
         return WFQ_ERR_INVALID_ARG;
     cudaStream_t st = as_stream(stream);
     cudaError_t e = wfq::launch_input_transform(*plan, x_dev, st);
-    if (e == cudaSuccess) e = wfq::launch_gemm(*plan, nullptr, st);
-    if (e == cudaSuccess) e = wfq::launch_output_transform(*plan, y_dev, st);
+    if (e == cudaSuccess) e = wfq::launch_gemm(*plan, nullptr, st, true);
+    if (e == cudaSuccess) e = wfq::launch_output_transform(*plan, y_dev, st, true);
     return cuda_status(e);
 }
 
@@ -294,7 +301,7 @@ wfq_status_t wfq_debug_get(wfq_plan_t *plan, wfq_buffer_t which, void **dev_ptr,
             *dev_ptr = plan->ws.Xq; *bytes = (size_t)g.P * g.T * g.C; return WFQ_OK;
         case WFQ_BUF_SX:
             if (!plan->has_workspace) return WFQ_ERR_NOT_PREPARED;
-            *dev_ptr = plan->ws.sX; *bytes = (size_t)g.P * g.G * g.T * sizeof(float); return WFQ_OK;
+            *dev_ptr = plan->ws.sX; *bytes = (size_t)g.P * g.G * g.Ts * sizeof(float); return WFQ_OK;
         case WFQ_BUF_Y:
             if (!plan->has_workspace) return WFQ_ERR_NOT_PREPARED;
             *dev_ptr = plan->ws.Y; *bytes = (size_t)g.P * g.K * g.Tp * sizeof(float); return WFQ_OK;
@@ -303,7 +310,7 @@ wfq_status_t wfq_debug_get(wfq_plan_t *plan, wfq_buffer_t which, void **dev_ptr,
             *dev_ptr = plan->Wq; *bytes = (size_t)g.P * g.K * g.C; return WFQ_OK;
         case WFQ_BUF_SW:
             if (!plan->prepared) return WFQ_ERR_NOT_PREPARED;
-            *dev_ptr = plan->sW; *bytes = (size_t)g.P * g.G * g.K * sizeof(float); return WFQ_OK;
+            *dev_ptr = plan->sW; *bytes = (size_t)g.P * g.G * g.Kp * sizeof(float); return WFQ_OK;
         case WFQ_BUF_STATUS:
             if (!plan->status) return WFQ_ERR_NOT_PREPARED;
             *dev_ptr = plan->status; *bytes = 4 * sizeof(int); return WFQ_OK;

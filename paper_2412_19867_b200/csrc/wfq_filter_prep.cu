@@ -58,9 +58,11 @@ __global__ void filter_transform_kernel(const float *__restrict__ w, float *__re
         }
 }
 
-// One thread per (p, k, g): abs-max of the group, scale, codes.
+// One thread per (p, k, g): abs-max of the group, scale, codes.  sW rows are k_pitch
+// floats apart.
 __global__ void filter_quantize_kernel(const float *__restrict__ w32, int8_t *__restrict__ Wq,
-                                       float *__restrict__ sW, int P, int K, int C, int gs)
+                                       float *__restrict__ sW, int P, int K, int C, int gs,
+                                       int k_pitch)
 {
     const int G = C / gs;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -77,7 +79,7 @@ __global__ void filter_quantize_kernel(const float *__restrict__ w32, int8_t *__
         scale = __fdiv_rn(amax, 127.f);
         inv = __fdiv_rn(127.f, amax);
     }
-    sW[((size_t)p * G + g) * K + k] = scale;
+    sW[((size_t)p * G + g) * k_pitch + k] = scale;
     for (int e = 0; e < gs; ++e) {
         int q = __float2int_rn(__fmul_rn(src[e], inv));
         q = max(-127, min(127, q));
@@ -106,7 +108,7 @@ cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *
         const int threads = 128;
         const unsigned blocks = (unsigned)((total + threads - 1) / threads);
         filter_quantize_kernel<<<blocks, threads, 0, stream>>>(scratch_w32, plan.Wq, plan.sW, g.P,
-                                                               g.K, g.C, g.gs);
+                                                               g.K, g.C, g.gs, g.Kp);
         return cudaGetLastError();
     }
 }
@@ -192,7 +194,7 @@ extern "C" wfq_status_t wfq_quantize_filters_static(const float *w_dev, int K, i
     {
         const long long total = (long long)P * K * (C / group_size);
         const unsigned blocks = (unsigned)((total + threads - 1) / threads);
-        filter_quantize_kernel<<<blocks, threads, 0, st>>>(w32, wq_dev, sw_dev, P, K, C, group_size);
+        filter_quantize_kernel<<<blocks, threads, 0, st>>>(w32, wq_dev, sw_dev, P, K, C, group_size, K);
         if (cudaGetLastError() != cudaSuccess) return WFQ_ERR_CUDA;
     }
     return WFQ_OK;

@@ -301,7 +301,7 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
                 *reinterpret_cast<uint4 *>(dst + c16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
             }
         }
-        sX[((size_t)p * g.G + g_base + grp) * g.T + t] = scale;
+        sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
     }
 }
 

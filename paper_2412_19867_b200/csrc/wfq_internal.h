@@ -19,14 +19,17 @@ enum WaitId : int {
     kWaitSmemFull = 2,    // MMA issuer waiting for TMA data
     kWaitTmemEmpty = 3,   // MMA issuer waiting for a drained accumulator
     kWaitTmemFull = 4,    // epilogue waiting for a finished accumulator
-    kWaitDrain = 5        // teardown waiting for copies in flight
+    kWaitDrain = 5,       // teardown waiting for copies in flight
+    kWaitScaleEmpty = 6,  // scale loader waiting for a free ring slot
+    kWaitScaleFull = 7    // epilogue waiting for a group's scales
 };
 
 // Geometry and scale tables handed to the kernels by value.
 struct Geometry {
     int N, C, K, H, W;
     int m, n, P;          // output tile, input tile, positions
-    int TH, TW, T, Tp;    // tiles per column/row, total, T rounded up to 32
+    int TH, TW, T, Tp;    // tiles per column/row, total, T rounded up to 32 (row pitch of Y)
+    int Ts, Kp;           // T and K rounded up to 128: row pitches of sX and sW
     int gs, G;            // channels per group, groups
 };
 
@@ -39,7 +42,7 @@ struct ScaleTables {
 
 struct Workspace {
     int8_t *Xq = nullptr;   // [P][T][C]
-    float *sX = nullptr;    // [P][G][T]
+    float *sX = nullptr;    // [P][G][Ts]
     float *Y = nullptr;     // [P][K][Tp]
     size_t xq_bytes = 0, sx_bytes = 0, y_bytes = 0, total = 0;
 };
@@ -57,7 +60,7 @@ struct wfq_plan {
 
     // plan-owned device memory
     int8_t *Wq = nullptr;      // [P][K][C]
-    float *sW = nullptr;       // [P][G][K]
+    float *sW = nullptr;       // [P][G][Kp]
     int *status = nullptr;     // int32[4]
     void *x_stage = nullptr;   // staging for wfq_conv_forward_host
     float *y_stage = nullptr;
@@ -68,6 +71,8 @@ struct wfq_plan {
     CUtensorMap tmap_xq;       // Xq as (C, T, P) bytes, 128B-swizzled boxes
     CUtensorMap tmap_wq;       // Wq as (C, K, P)
     bool tmap_xq_ok = false, tmap_wq_ok = false;
+    bool gemm_swap = false;    // contraction rows are output channels instead of tiles
+    int gemm_bn = 64;          // columns per unit of the contraction
 };
 
 namespace wfq {
@@ -77,15 +82,15 @@ namespace wfq {
 cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *scratch_w32,
                                cudaStream_t stream);
 cudaError_t launch_input_transform(const wfq_plan &plan, const void *x_dev, cudaStream_t stream);
-cudaError_t launch_gemm(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t stream);
-cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStream_t stream);
+cudaError_t launch_gemm(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t stream, bool pdl);
+cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStream_t stream, bool pdl);
 
 // Builds a 3-D byte tensor map (inner extent `inner`, rows, planes) with a
 // (128, box_rows, 1) box and 128-byte swizzle.  Returns false on failure.
 bool encode_tmap_bytes3d(CUtensorMap *map, const void *base, int inner, int rows, int planes,
                          int box_rows);
 
-int gemm_block_n();   // output channels per CTA tile of the contraction kernel
-int gemm_block_m();   // tiles per CTA tile (128)
+int gemm_block_m();   // rows per unit of the contraction kernel (128)
+void gemm_choose(const Geometry &g, bool *swap, int *bn);
 
 }  // namespace wfq

@@ -4,6 +4,7 @@
 // neighbouring lanes are contiguous in y[N][K][H][W].  Memory-bound: P*4 bytes read
 // and m*m*4 bytes written per thread against ~150 flops.
 #include "wfq_internal.h"
+#include "wfq_ptx.cuh"
 
 namespace wfq {
 namespace {
@@ -48,6 +49,7 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
     constexpr int NN = M + 2;
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
+    ptx::grid_dependency_wait();   // Y comes from the kernel launched before this one
     if (t >= g.T) return;
 
     const size_t plane = (size_t)g.K * g.Tp;
@@ -100,16 +102,22 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
 
 }  // namespace
 
-cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStream_t stream)
+cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStream_t stream, bool pdl)
 {
     const Geometry &g = plan.geo;
     const int threads = 128;
-    dim3 grid((g.T + threads - 1) / threads, g.K);
-    if (g.m == 4)
-        output_transform_kernel<4><<<grid, threads, 0, stream>>>(plan.ws.Y, y_dev, g, plan.tables);
-    else
-        output_transform_kernel<6><<<grid, threads, 0, stream>>>(plan.ws.Y, y_dev, g, plan.tables);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((g.T + threads - 1) / threads, g.K);
+    cfg.blockDim = dim3(threads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    const float *Y = plan.ws.Y;
+    if (g.m == 4) return cudaLaunchKernelEx(&cfg, output_transform_kernel<4>, Y, y_dev, g, plan.tables);
+    return cudaLaunchKernelEx(&cfg, output_transform_kernel<6>, Y, y_dev, g, plan.tables);
 }
 
 }  // namespace wfq

@@ -21,6 +21,13 @@ def make_conv(layer, tensors=None, device="cuda:0"):
     return conv, (x, w, sB, sG)
 
 
+def padded(a, pitch):
+    """Zero-pad the last axis of a float array to `pitch` (the row pitch of sX / sW)."""
+    out = np.zeros(a.shape[:-1] + (pitch,), dtype=np.float32)
+    out[..., :a.shape[-1]] = a
+    return out
+
+
 def codes_close(got, want):
     """int8 tensors: identical except at most CODE_MISMATCH_RATE of elements off by one."""
     got = np.asarray(got).astype(np.int16)
@@ -58,20 +65,22 @@ def check_layer_all_levels(layer, tensors=None, final_tol=FINAL_TOL):
 
     # offline filter path
     report["wq_rate"] = codes_close(conv.buffer(b.WFQ_BUF_WQ).cpu().numpy(), ref.Wq)
-    scales_close(conv.buffer(b.WFQ_BUF_SW).cpu().numpy(), ref.sW.transpose(0, 2, 1), rtol=1e-6)
+    sw_all = conv.buffer(b.WFQ_BUF_SW).cpu().numpy()
+    scales_close(sw_all[:, :, :layer.K], ref.sW.transpose(0, 2, 1), rtol=1e-6)
+    assert not sw_all[:, :, layer.K:].any(), "sW padding columns must be zero"
 
     # stage 1: fused input transform + quantize
     xd = torch.from_numpy(x).to(dev)
     b.wfq_input_transform_quantize(conv.plan, xd.data_ptr(), conv._stream())
     torch.cuda.synchronize()
     report["xq_rate"] = codes_close(conv.buffer(b.WFQ_BUF_XQ).cpu().numpy(), ref.Xq)
-    scales_close(conv.buffer(b.WFQ_BUF_SX).cpu().numpy(), ref.sX.transpose(0, 2, 1))
+    scales_close(conv.buffer(b.WFQ_BUF_SX).cpu().numpy()[:, :, :conv.T], ref.sX.transpose(0, 2, 1))
 
     # identical int8 operands from here on: the oracle's codes and scales
     conv.write_buffer(b.WFQ_BUF_XQ, torch.from_numpy(ref.Xq))
-    conv.write_buffer(b.WFQ_BUF_SX, torch.from_numpy(np.ascontiguousarray(ref.sX.transpose(0, 2, 1))))
+    conv.write_buffer(b.WFQ_BUF_SX, torch.from_numpy(padded(ref.sX.transpose(0, 2, 1), conv.Ts)))
     conv.write_buffer(b.WFQ_BUF_WQ, torch.from_numpy(ref.Wq))
-    conv.write_buffer(b.WFQ_BUF_SW, torch.from_numpy(np.ascontiguousarray(ref.sW.transpose(0, 2, 1))))
+    conv.write_buffer(b.WFQ_BUF_SW, torch.from_numpy(padded(ref.sW.transpose(0, 2, 1), conv.Kp)))
 
     # level 1: int32 group accumulators, bit exact
     acc = torch.empty(ref.acc.shape, dtype=torch.int32, device=dev)

@@ -63,9 +63,10 @@ def test_workspace_size_and_order_of_calls(lib):
     assert st == b.WFQ_OK
     n, P = m + 2, (m + 2) ** 2
     T = N * (-(-H // m)) * (-(-W // m))
-    Tp = (T + 31) // 32 * 32
+    Tp = (T + 31) // 32 * 32            # row pitch of Y
+    Ts = (T + 127) // 128 * 128         # row pitch of sX
     up = lambda v: (v + 1023) // 1024 * 1024
-    want = up(P * T * C) + up(P * (C // gs) * T * 4) + up(P * K * Tp * 4)
+    want = up(P * T * C) + up(P * (C // gs) * Ts * 4) + up(P * K * Tp * 4)
     assert lib.wfq_plan_workspace_bytes(plan) == want
     assert lib.wfq_plan_workspace_bytes(None) == 0
     # nothing may run before workspace + filters exist

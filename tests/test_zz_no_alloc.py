@@ -23,7 +23,7 @@ def _both_ways(layer):
     from tests.gpu_util import make_conv, codes_close, scales_close
     conv, (x, w, sB, sG) = make_conv(layer)                    # wfq_prepare_filters
     want_q = conv.buffer(b.WFQ_BUF_WQ).cpu().numpy()
-    want_s = conv.buffer(b.WFQ_BUF_SW).cpu().numpy()
+    want_s = conv.buffer(b.WFQ_BUF_SW).cpu().numpy()[:, :, :layer.K]     # rows are padded to 128
     wd = torch.from_numpy(w).cuda()
     # outputs pre-filled so that unwritten elements would show
     got_q = torch.full(want_q.shape, 99, dtype=torch.int8, device="cuda")
