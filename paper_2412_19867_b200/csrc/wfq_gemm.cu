@@ -2,23 +2,34 @@
 //   for every position p:  Y_p[t][k] = sum_g sX[p,g,t] * sW[p,g,k] * acc_g[t][k],
 //   acc_g[t][k] = sum_{c in g} Xq_p[t][c] * Wq_p[k][c]     (int8 x int8 -> int32)
 //
-// Persistent, warp-specialised sm_100a kernel, one CTA per SM.  A unit of work is
+// Persistent, warp-specialised sm_100a kernel, two CTAs per SM.  A unit of work is
 // (position p, block of 128 rows, block of BN columns).  "Rows" are the 128 TMEM lanes
 // of the accumulator: tiles in the normal orientation, output channels in the swapped
 // one (used when there are few tiles, so that all 128 lanes carry real work); columns
 // are the other of the two.  Both operands are K-major int8 (channels contiguous).
-//   warp 0       TMA producer: 128 x 128 B of the row operand and BN x 128 B of the
-//                column operand per stage (128-byte swizzle), ring of NSTAGES mbarriers
-//   warp 1       allocates TMEM; one lane issues tcgen05.mma kind::i8 (M=128, N=BN,
-//                K=32 per instruction).  Every channel group accumulates into its own
-//                TMEM buffer (ring of NBUF) and is committed to an mbarrier when done
-//   warp 2       scale loader: per group, 128 row scales and BN column scales go to a
-//                shared-memory ring with two bulk copies
-//   warps 4-19   epilogue: quarter = warp % 4 selects the 32 TMEM lanes the warp may
-//                read, (warp - 4) / 4 selects BN/4 of the columns.  tcgen05.ld the
-//                finished int32 group sums, release the buffer, convert and scale
-//                into fp32 registers; after the last group write Y[p][k][t]
-// The tensor pipe therefore runs groups g+1.. while the ALUs promote group g.
+//
+// Every mbarrier hand-over costs the thread that makes it a few hundred cycles, so the
+// roles synchronise per *chunk* of up to CG channel groups (128 channels when the group
+// size divides 128), not per group.  A chunk owns one TMEM slot of 128 columns (its
+// groups side by side, BN columns each) and one slot of the scale ring.
+//   warp 0   TMA producer: 128 x 128 B of the row operand and BN x 128 B of the column
+//            operand per stage (128-byte swizzle), ring of NSTAGES
+//   warp 1   allocates TMEM; one lane issues tcgen05.mma kind::i8 (M=128, N=BN, K=32 per
+//            instruction): waits for a stage and, at the start of a chunk, for its TMEM
+//            slot; commits the stage back to the producer and the chunk to the epilogue
+//   warp 2   scale loader: per chunk, 128 row scales and BN column scales per group into
+//            the chunk's scale slot (bulk copies)
+//   warps 4-7   epilogue: warp % 4 selects the 32 TMEM lanes the warp may read; each warp
+//            handles all BN columns of its lanes.  Per chunk: wait for accumulators and
+//            scales, then per group tcgen05.ld the int32 sums, convert and scale into fp32
+//            registers (packed f32x2 multiply / fma), release the slot; after the last
+//            chunk of a unit write Y[p][k][t].
+// The second CTA of the SM runs the same pipeline on other units, which hides the
+// hand-over latencies and overlaps one CTA's output stores with the other's arithmetic.
+// Only four epilogue warps per CTA on purpose: the warp schedulers share issue slots
+// evenly among ready warps, so every additional arithmetic warp slows the three
+// single-purpose warps whose few instructions sit on the critical path (measured:
+// 8 epilogue warps per CTA were 15-25 % slower).
 // Every wait is bounded; on expiry the CTA records where, stops, drains and frees TMEM.
 #include "wfq_internal.h"
 #include "wfq_ptx.cuh"
@@ -30,22 +41,22 @@ namespace {
 constexpr int BM = 128;        // rows per unit (MMA M, TMEM lanes)
 constexpr int BK = 128;        // bytes (= int8 channels) per pipeline stage
 constexpr int UK = 32;         // channels per MMA instruction
-constexpr int NSTAGES = 7;
-constexpr int NBUF = 8;        // TMEM accumulator buffers
-constexpr int NSC = 16;        // scale ring slots (one group each)
+constexpr int NSTAGES = 4;     // shared-memory operand stages
+constexpr int NSLOT = 2;       // TMEM / scale slots (chunks in flight)
+constexpr int SLOT_COLS = 128; // TMEM columns per slot
+constexpr int TMEM_COLS = NSLOT * SLOT_COLS;
 constexpr int A_BYTES = BM * BK;
-constexpr int NUM_EPI_WARPS = 16;
+constexpr int NUM_EPI_WARPS = 4;
 constexpr int FIRST_EPI_WARP = 4;
 constexpr int NUM_THREADS = 32 * (FIRST_EPI_WARP + NUM_EPI_WARPS);
 constexpr long long WAIT_CYCLES = 2000000000LL;   // ~1 s at 2 GHz
 
 struct Shared {
-    uint64_t full[NSTAGES];
-    uint64_t empty[NSTAGES];
-    uint64_t tmem_full[NBUF];
-    uint64_t tmem_empty[NBUF];
-    uint64_t scale_full[NSC];
-    uint64_t scale_empty[NSC];
+    uint64_t full[NSTAGES];        // operands of a stage have landed
+    uint64_t empty[NSTAGES];       // the MMAs reading a stage have completed
+    uint64_t acc_full[NSLOT];      // the MMAs of a chunk have completed
+    uint64_t slot_free[NSLOT];     // all epilogue warps are done with a chunk
+    uint64_t scale_full[NSLOT];    // the scales of a chunk have landed
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -54,40 +65,47 @@ template <int BN>
 struct Cfg {
     static constexpr int B_BYTES = BN * BK;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int SCALE_FLOATS = BM + BN;              // per ring slot
-    static constexpr int TMEM_COLS = NBUF * BN;               // 512 or 256: a power of two
+    static constexpr int CG_MAX = SLOT_COLS / BN;             // groups per chunk at most
+    static constexpr int GROUP_SCALE_FLOATS = BM + BN;        // row scales, then column scales
+    static constexpr int SLOT_SCALE_FLOATS = CG_MAX * GROUP_SCALE_FLOATS;
     static constexpr int CW = BN / (NUM_EPI_WARPS / 4);       // columns per epilogue warp
     static constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)NSTAGES * STAGE_BYTES +
-                                         (size_t)NSC * SCALE_FLOATS * sizeof(float) + sizeof(Shared);
+                                         (size_t)NSLOT * SLOT_SCALE_FLOATS * sizeof(float) + sizeof(Shared);
 };
 
 // Bounded mbarrier wait.  Returns false (and records `where`) on timeout or when
-// another role of this CTA already gave up.
+// another role of this CTA already gave up.  The loop body is the bare try_wait (which
+// suspends the thread in hardware for a while); clock and abort flag are looked at
+// every 1024 tries.
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Shared *sh, int *status,
                                              int where)
 {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (true) {
+    long long t0 = 0;
+#pragma unroll 1
+    for (uint32_t it = 1;; ++it) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
-        if (sh->abort) return false;
-        if (clock64() - t0 > WAIT_CYCLES) {
-            sh->abort = 1;
-            if (atomicCAS(status, 0, (int)WFQ_ERR_TIMEOUT) == 0) {
-                status[1] = where;
-                status[2] = (int)blockIdx.x;
-                status[3] = (int)parity;
+        if ((it & 1023u) == 0) {
+            if (sh->abort) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > WAIT_CYCLES) {
+                sh->abort = 1;
+                if (atomicCAS(status, 0, (int)WFQ_ERR_TIMEOUT) == 0) {
+                    status[1] = where;
+                    status[2] = (int)blockIdx.x;
+                    status[3] = (int)parity;
+                }
+                return false;
             }
-            return false;
         }
     }
 }
 
-template <int N>
-__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[N])
+// Bounded wait for copies that may still be in flight when a role gives up.
+__device__ __forceinline__ void drain(uint32_t bar, uint32_t parity)
 {
-    if constexpr (N == 16) ptx::tmem_ld_x16(taddr, r);
-    else ptx::tmem_ld_x8(taddr, r);
+    const long long t0 = clock64();
+    while (!ptx::mbar_try_wait(bar, parity) && clock64() - t0 < WAIT_CYCLES / 16) { }
 }
 
 struct GemmArgs {
@@ -95,13 +113,14 @@ struct GemmArgs {
     const float *col_scale;   // [P][G][col_pitch]: sW (normal) or sX (swapped)
     int row_pitch, col_pitch;
     int rows, cols;           // valid rows / columns: (T, K) normal, (K, T) swapped
+    int cg;                   // groups per chunk
     float *Y;                 // [P][K][Tp]
     int32_t *acc_dump;        // [P][T][K][G] or null
     int *status;
 };
 
 template <int BN, bool SWAP, bool DUMP>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(NUM_THREADS, 2)
 gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     GemmArgs a, Geometry g)
 {
@@ -112,13 +131,15 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     unsigned char *tiles = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     float *scales = reinterpret_cast<float *>(tiles + (size_t)NSTAGES * C::STAGE_BYTES);
-    Shared *sh = reinterpret_cast<Shared *>(scales + (size_t)NSC * C::SCALE_FLOATS);
+    Shared *sh = reinterpret_cast<Shared *>(scales + (size_t)NSLOT * C::SLOT_SCALE_FLOATS);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int MT = (a.rows + BM - 1) / BM, NT = (a.cols + BN - 1) / BN;
     const int units = g.P * MT * NT;
     const int KB = (g.C + BK - 1) / BK;          // stages per unit
     const int gs_steps = g.gs / UK;              // MMAs per group
+    const int cg = a.cg;                         // groups per chunk
+    const int nchunk = (g.G + cg - 1) / cg;      // chunks per unit
     int *status = a.status;
 
     if (threadIdx.x == 0) {
@@ -126,19 +147,16 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
         }
-        for (int b = 0; b < NBUF; ++b) {
-            ptx::mbar_init(ptx::smem_u32(&sh->tmem_full[b]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh->tmem_empty[b]), NUM_EPI_WARPS);
-        }
-        for (int s = 0; s < NSC; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&sh->scale_full[s]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh->scale_empty[s]), NUM_EPI_WARPS);
+        for (int b = 0; b < NSLOT; ++b) {
+            ptx::mbar_init(ptx::smem_u32(&sh->acc_full[b]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh->slot_free[b]), NUM_EPI_WARPS);
+            ptx::mbar_init(ptx::smem_u32(&sh->scale_full[b]), 1);
         }
         sh->abort = 0;
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), C::TMEM_COLS);
+        ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), TMEM_COLS);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before();
@@ -151,112 +169,143 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
+        // All 32 lanes walk the loop and wait together; lane 0 alone issues the copies.
+        // (A warp whose other lanes sit at the final block barrier while one lane works
+        // gets scheduled far too rarely.)
         if (lane == 0) {
             ptx::prefetch_tmap(&tmA);
             ptx::prefetch_tmap(&tmB);
-            int stage = 0;
-            uint32_t phase = 0;
-            long long issued = 0;
-            bool ok = true;
-            for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-                const int nt = u % NT, mt = (u / NT) % MT, p = u / (NT * MT);
-                for (int kb = 0; kb < KB; ++kb) {
-                    if (!wait_bounded(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, sh, status,
-                                      kWaitSmemEmpty)) { ok = false; break; }
+        }
+        int stage = 0;
+        uint32_t phase = 0;
+        long long issued = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+            const int nt = u % NT, mt = (u / NT) % MT, p = u / (NT * MT);
+            for (int kb = 0; kb < KB; ++kb) {
+                ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, sh,
+                                                          status, kWaitSmemEmpty));
+                if (!ok) break;
+                if (lane == 0) {
                     const uint32_t bar = ptx::smem_u32(&sh->full[stage]);
                     const uint32_t a_dst = ptx::smem_u32(tiles + (size_t)stage * C::STAGE_BYTES);
                     ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
                     ptx::tma_load_3d(a_dst, &tmA, bar, kb * BK, mt * BM, p);
                     ptx::tma_load_3d(a_dst + A_BYTES, &tmB, bar, kb * BK, nt * BN, p);
-                    ++issued;
-                    if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
                 }
+                __syncwarp();
+                ++issued;
+                if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
             }
-            if (!ok) {
-                // give copies still in flight a bounded time to land before the CTA exits
-                int s = stage;
-                uint32_t ph = phase;
-                const long long n = issued < NSTAGES ? issued : NSTAGES;
-                for (long long i = 0; i < n; ++i) {
-                    if (--s < 0) { s = NSTAGES - 1; ph ^= 1u; }
-                    const long long t0 = clock64();
-                    while (!ptx::mbar_try_wait(ptx::smem_u32(&sh->full[s]), ph) &&
-                           clock64() - t0 < WAIT_CYCLES / 16) { }
-                }
+        }
+        if (!ok) {
+            // give copies still in flight a bounded time to land before the CTA exits
+            int s = stage;
+            uint32_t ph = phase;
+            const long long n = issued < NSTAGES ? issued : NSTAGES;
+            for (long long i = 0; i < n; ++i) {
+                if (--s < 0) { s = NSTAGES - 1; ph ^= 1u; }
+                drain(ptx::smem_u32(&sh->full[s]), ph);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
-            int stage = 0, buf = 0;
-            uint32_t phase = 0, tphase = 0;
-            bool ok = true;
-            for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-                int step_in_group = 0;
-                for (int kb = 0; kb < KB && ok; ++kb) {
-                    if (!wait_bounded(ptx::smem_u32(&sh->full[stage]), phase, sh, status, kWaitSmemFull)) {
-                        ok = false; break;
+        // The warp stays converged; lane 0 issues every MMA and commit.  Its instructions
+        // form one dependent chain, so the descriptors are advanced with 32-bit adds and
+        // the accumulate flag is a constant of the instruction.
+        constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
+        constexpr uint32_t dhi = ptx::smem_desc_sw128_hi();
+        const uint32_t tiles_lo = ptx::smem_desc_sw128_lo(ptx::smem_u32(tiles));
+        const int chunk_steps = cg * gs_steps;       // MMAs per full chunk
+        int stage = 0, slot = 0;
+        uint32_t phase = 0, sphase = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+            int step = 0;          // MMA step within the chunk
+            int in_group = 0;      // MMA step within the group
+            uint32_t dcol = 0;     // TMEM column of the current group
+            for (int kb = 0; kb < KB && ok; ++kb) {
+                ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->full[stage]), phase, sh, status,
+                                                          kWaitSmemFull));
+                if (!ok) break;
+                ptx::tc_fence_after();
+                // a 32-byte step along K inside the swizzled rows is +2 in the address field
+                const uint32_t a_lo = tiles_lo + (uint32_t)(stage * (C::STAGE_BYTES >> 4));
+                const uint32_t b_lo = a_lo + (uint32_t)(A_BYTES >> 4);
+                const int nslice = min(BK, g.C - kb * BK) / UK;
+                for (int s = 0; s < nslice; ++s) {
+                    if (step == 0) {
+                        // start of a chunk: its TMEM slot must have been drained
+                        ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->slot_free[slot]),
+                                                                  sphase ^ 1u, sh, status, kWaitTmemEmpty));
+                        if (!ok) break;
+                        ptx::tc_fence_after();
+                        dcol = tmem_base + (uint32_t)(slot * SLOT_COLS);
                     }
-                    ptx::tc_fence_after();
-                    const uint32_t a_addr = ptx::smem_u32(tiles + (size_t)stage * C::STAGE_BYTES);
-                    const uint64_t a_desc = ptx::smem_desc_sw128(a_addr);
-                    const uint64_t b_desc = ptx::smem_desc_sw128(a_addr + A_BYTES);
-                    const int nslice = min(BK, g.C - kb * BK) / UK;
-                    for (int s = 0; s < nslice; ++s) {
-                        if (step_in_group == 0) {
-                            if (!wait_bounded(ptx::smem_u32(&sh->tmem_empty[buf]), tphase ^ 1u, sh,
-                                              status, kWaitTmemEmpty)) { ok = false; break; }
-                            ptx::tc_fence_after();
-                        }
-                        // advancing the start address by 32 bytes (>>4 = 2) walks along K
-                        // inside the swizzled 128-byte rows
-                        ptx::umma_i8(tmem_base + (uint32_t)(buf * BN), a_desc + (uint64_t)(2 * s),
-                                     b_desc + (uint64_t)(2 * s), idesc, step_in_group ? 1u : 0u);
-                        if (++step_in_group == gs_steps) {
-                            ptx::umma_commit(ptx::smem_u32(&sh->tmem_full[buf]));
-                            step_in_group = 0;
-                            if (++buf == NBUF) { buf = 0; tphase ^= 1u; }
-                        }
+                    if (lane == 0) {
+                        if (in_group) ptx::umma_i8_lo<true>(dcol, a_lo + 2 * s, b_lo + 2 * s, dhi, idesc);
+                        else ptx::umma_i8_lo<false>(dcol, a_lo + 2 * s, b_lo + 2 * s, dhi, idesc);
                     }
-                    ptx::umma_commit(ptx::smem_u32(&sh->empty[stage]));
-                    if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
+                    ++step;
+                    if (++in_group == gs_steps) { in_group = 0; dcol += BN; }
+                    if (step == chunk_steps) {
+                        if (lane == 0) ptx::umma_commit(ptx::smem_u32(&sh->acc_full[slot]));
+                        step = 0;
+                        if (++slot == NSLOT) { slot = 0; sphase ^= 1u; }
+                    }
                 }
+                if (!ok) break;
+                if (lane == 0) ptx::umma_commit(ptx::smem_u32(&sh->empty[stage]));
+                __syncwarp();
+                if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (ok && step != 0) {
+                // the last chunk of the unit has fewer groups than a full one
+                if (lane == 0) ptx::umma_commit(ptx::smem_u32(&sh->acc_full[slot]));
+                __syncwarp();
+                if (++slot == NSLOT) { slot = 0; sphase ^= 1u; }
             }
         }
     } else if (warp == 2) {
         // ---------------- scale loader ----------------
-        if (lane == 0 && !DUMP) {
+        if (!DUMP) {
             int slot = 0;
             uint32_t sphase = 0;
             long long issued = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
                 const int nt = u % NT, mt = (u / NT) % MT, p = u / (NT * MT);
-                for (int grp = 0; grp < g.G; ++grp) {
-                    if (!wait_bounded(ptx::smem_u32(&sh->scale_empty[slot]), sphase ^ 1u, sh, status,
-                                      kWaitScaleEmpty)) { ok = false; break; }
+                for (int ch = 0; ch < nchunk; ++ch) {
+                    const int g0 = ch * cg, ng = min(cg, g.G - g0);
+                    ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->slot_free[slot]), sphase ^ 1u,
+                                                              sh, status, kWaitScaleEmpty));
+                    if (!ok) break;
                     const uint32_t bar = ptx::smem_u32(&sh->scale_full[slot]);
-                    const uint32_t dst = ptx::smem_u32(scales + (size_t)slot * C::SCALE_FLOATS);
-                    ptx::mbar_arrive_expect_tx(bar, C::SCALE_FLOATS * 4);
-                    ptx::bulk_load(dst, a.row_scale + ((size_t)p * g.G + grp) * a.row_pitch + mt * BM,
-                                   BM * 4, bar);
-                    ptx::bulk_load(dst + BM * 4,
-                                   a.col_scale + ((size_t)p * g.G + grp) * a.col_pitch + nt * BN,
-                                   BN * 4, bar);
+                    const uint32_t dst = ptx::smem_u32(scales + (size_t)slot * C::SLOT_SCALE_FLOATS);
+                    if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)(ng * C::GROUP_SCALE_FLOATS * 4));
+                    __syncwarp();
+                    // lane j copies the row scales of group j, lane 4 + j its column scales
+                    if (lane < 8 && (lane & 3) < ng) {
+                        const int j = lane & 3;
+                        const size_t pg = (size_t)p * g.G + g0 + j;
+                        const uint32_t d = dst + (uint32_t)(j * C::GROUP_SCALE_FLOATS * 4);
+                        if (lane < 4)
+                            ptx::bulk_load(d, a.row_scale + pg * a.row_pitch + mt * BM, BM * 4, bar);
+                        else
+                            ptx::bulk_load(d + BM * 4, a.col_scale + pg * a.col_pitch + nt * BN, BN * 4, bar);
+                    }
+                    __syncwarp();
                     ++issued;
-                    if (++slot == NSC) { slot = 0; sphase ^= 1u; }
+                    if (++slot == NSLOT) { slot = 0; sphase ^= 1u; }
                 }
             }
             if (!ok) {
                 int s = slot;
                 uint32_t ph = sphase;
-                const long long n = issued < NSC ? issued : NSC;
+                const long long n = issued < NSLOT ? issued : NSLOT;
                 for (long long i = 0; i < n; ++i) {
-                    if (--s < 0) { s = NSC - 1; ph ^= 1u; }
-                    const long long t0 = clock64();
-                    while (!ptx::mbar_try_wait(ptx::smem_u32(&sh->scale_full[s]), ph) &&
-                           clock64() - t0 < WAIT_CYCLES / 16) { }
+                    if (--s < 0) { s = NSLOT - 1; ph ^= 1u; }
+                    drain(ptx::smem_u32(&sh->scale_full[s]), ph);
                 }
             }
         }
@@ -264,8 +313,9 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // ---------------- epilogue ----------------
         const int quarter = warp & 3;                         // TMEM lanes this warp may read
         const int c0 = ((warp - FIRST_EPI_WARP) >> 2) * CW;   // first column of this warp
-        int buf = 0, slot = 0;
-        uint32_t tphase = 0, sphase = 0;
+        const uint32_t tmem_warp = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0;
+        int slot = 0;
+        uint32_t sphase = 0;
         bool ok = true;
         for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
             const int nt = u % NT, mt = (u / NT) % MT, p = u / (NT * MT);
@@ -274,58 +324,69 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // warp-uniform: does this warp own any valid row and column of the unit?
             const bool active = (mt * BM + quarter * 32 < a.rows) && (col0 < a.cols);
             const bool row_ok = row < a.rows;
-            float acc[CW];
+            float2 acc[CW / 2];
 #pragma unroll
-            for (int j = 0; j < CW; ++j) acc[j] = 0.f;
-            for (int grp = 0; grp < g.G; ++grp) {
-                if (!wait_bounded(ptx::smem_u32(&sh->tmem_full[buf]), tphase, sh, status, kWaitTmemFull)) {
+            for (int j = 0; j < CW / 2; ++j) acc[j] = make_float2(0.f, 0.f);
+
+            for (int ch = 0; ch < nchunk && ok; ++ch) {
+                const int g0 = ch * cg, ng = min(cg, g.G - g0);
+                if (!wait_bounded(ptx::smem_u32(&sh->acc_full[slot]), sphase, sh, status, kWaitTmemFull)) {
                     ok = false; break;
                 }
-                uint32_t r[CW];
+                if constexpr (!DUMP) {
+                    if (!wait_bounded(ptx::smem_u32(&sh->scale_full[slot]), sphase, sh, status,
+                                      kWaitScaleFull)) { ok = false; break; }
+                }
                 if (active) {
                     ptx::tc_fence_after();
-                    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) +
-                                           (uint32_t)(buf * BN + c0);
-                    tmem_ld_cols<CW>(taddr, r);
-                    ptx::tmem_ld_wait();
-                    ptx::tc_fence_before();
-                }
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->tmem_empty[buf]));
-                if (++buf == NBUF) { buf = 0; tphase ^= 1u; }
-
-                if constexpr (DUMP) {
-                    if (active && row_ok) {
+                    const float *sc = scales + (size_t)slot * C::SLOT_SCALE_FLOATS;
+                    for (int j = 0; j < ng; ++j) {
+                        const uint32_t taddr = tmem_warp + (uint32_t)(slot * SLOT_COLS + j * BN);
+                        const float rs = sc[j * C::GROUP_SCALE_FLOATS + quarter * 32 + lane];
+                        const float2 rs2 = make_float2(rs, rs);
+                        const float4 *cs4 = reinterpret_cast<const float4 *>(
+                            sc + j * C::GROUP_SCALE_FLOATS + BM + c0);
 #pragma unroll
-                        for (int j = 0; j < CW; ++j) {
-                            const int col = col0 + j;
-                            if (col < a.cols) {
-                                const size_t t = SWAP ? col : row, k = SWAP ? row : col;
-                                a.acc_dump[(((size_t)p * g.T + t) * g.K + k) * g.G + grp] = (int32_t)r[j];
+                        for (int h = 0; h < CW / 16; ++h) {          // 16 columns at a time
+                            uint32_t r[16];
+                            ptx::tmem_ld_x16(taddr + (uint32_t)(16 * h), r);
+                            ptx::tmem_ld_wait();
+                            if constexpr (DUMP) {
+                                if (row_ok) {
+#pragma unroll
+                                    for (int i = 0; i < 16; ++i) {
+                                        const int col = col0 + 16 * h + i;
+                                        if (col < a.cols) {
+                                            const size_t t = SWAP ? col : row, k = SWAP ? row : col;
+                                            a.acc_dump[(((size_t)p * g.T + t) * g.K + k) * g.G + g0 + j] =
+                                                (int32_t)r[i];
+                                        }
+                                    }
+                                }
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const float4 cs = cs4[4 * h + q];
+                                    float2 f0 = make_float2(__int2float_rn((int32_t)r[4 * q + 0]),
+                                                            __int2float_rn((int32_t)r[4 * q + 1]));
+                                    float2 f1 = make_float2(__int2float_rn((int32_t)r[4 * q + 2]),
+                                                            __int2float_rn((int32_t)r[4 * q + 3]));
+                                    f0 = __fmul2_rn(f0, rs2);
+                                    f1 = __fmul2_rn(f1, rs2);
+                                    acc[8 * h + 2 * q] = __ffma2_rn(f0, make_float2(cs.x, cs.y), acc[8 * h + 2 * q]);
+                                    acc[8 * h + 2 * q + 1] =
+                                        __ffma2_rn(f1, make_float2(cs.z, cs.w), acc[8 * h + 2 * q + 1]);
+                                }
                             }
                         }
                     }
-                } else {
-                    if (!wait_bounded(ptx::smem_u32(&sh->scale_full[slot]), sphase, sh, status,
-                                      kWaitScaleFull)) { ok = false; break; }
-                    if (active) {
-                        const float *sc = scales + (size_t)slot * C::SCALE_FLOATS;
-                        const float rs = sc[quarter * 32 + lane];
-                        const float4 *cs4 = reinterpret_cast<const float4 *>(sc + BM + c0);
-#pragma unroll
-                        for (int j4 = 0; j4 < CW / 4; ++j4) {
-                            const float4 cs = cs4[j4];
-                            acc[4 * j4 + 0] = fmaf(__int2float_rn((int32_t)r[4 * j4 + 0]) * rs, cs.x, acc[4 * j4 + 0]);
-                            acc[4 * j4 + 1] = fmaf(__int2float_rn((int32_t)r[4 * j4 + 1]) * rs, cs.y, acc[4 * j4 + 1]);
-                            acc[4 * j4 + 2] = fmaf(__int2float_rn((int32_t)r[4 * j4 + 2]) * rs, cs.z, acc[4 * j4 + 2]);
-                            acc[4 * j4 + 3] = fmaf(__int2float_rn((int32_t)r[4 * j4 + 3]) * rs, cs.w, acc[4 * j4 + 3]);
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->scale_empty[slot]));
-                    if (++slot == NSC) { slot = 0; sphase ^= 1u; }
+                    ptx::tc_fence_before();
                 }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->slot_free[slot]));
+                if (++slot == NSLOT) { slot = 0; sphase ^= 1u; }
             }
+
             if constexpr (!DUMP) {
                 if (ok && active && row_ok) {
                     if constexpr (SWAP) {
@@ -335,13 +396,15 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         for (int j4 = 0; j4 < CW / 4; ++j4)
                             if (col0 + 4 * j4 + 3 < g.Tp)
                                 *reinterpret_cast<float4 *>(dst + 4 * j4) =
-                                    make_float4(acc[4 * j4], acc[4 * j4 + 1], acc[4 * j4 + 2], acc[4 * j4 + 3]);
+                                    make_float4(acc[2 * j4].x, acc[2 * j4].y, acc[2 * j4 + 1].x, acc[2 * j4 + 1].y);
                     } else {
                         // row = tile: lanes write consecutive t of one Y[p][k][:] row
                         float *dst = a.Y + ((size_t)p * g.K + col0) * g.Tp + row;
 #pragma unroll
-                        for (int j = 0; j < CW; ++j)
-                            if (col0 + j < a.cols) dst[(size_t)j * g.Tp] = acc[j];
+                        for (int j = 0; j < CW / 2; ++j) {
+                            if (col0 + 2 * j < a.cols) dst[(size_t)(2 * j) * g.Tp] = acc[j].x;
+                            if (col0 + 2 * j + 1 < a.cols) dst[(size_t)(2 * j + 1) * g.Tp] = acc[j].y;
+                        }
                     }
                 }
             }
@@ -352,7 +415,7 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
+        ptx::tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -368,12 +431,17 @@ cudaError_t launch_variant(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t
     a.col_pitch = SWAP ? g.Ts : g.Kp;
     a.rows = SWAP ? g.K : g.T;
     a.cols = SWAP ? g.T : g.K;
+    // groups per chunk: as many whole groups as fit into 128 channels (one stage) and
+    // into one TMEM slot; group sizes that do not divide 128 get one group per chunk
+    a.cg = 1;
+    if (BK % g.gs == 0) a.cg = BK / g.gs < C::CG_MAX ? BK / g.gs : C::CG_MAX;
     a.Y = plan.ws.Y;
     a.acc_dump = acc_dump;
     a.status = plan.status;
     const int MT = (a.rows + BM - 1) / BM, NT = (a.cols + BN - 1) / BN;
     const int units = g.P * MT * NT;
-    const int grid = units < plan.sm_count ? units : plan.sm_count;
+    const int slots = 2 * plan.sm_count;          // two CTAs per SM
+    const int grid = units < slots ? units : slots;
     auto kern = gemm_dequant_kernel<BN, SWAP, DUMP>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)C::SMEM_BYTES);

@@ -120,6 +120,30 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Same with the descriptors given as their low words (start address >> 4 plus the
+// fixed leading-offset field) over a common high word, and the accumulate flag as a
+// compile-time constant: the issuing thread runs a dependent instruction chain, so
+// every instruction saved per MMA shortens the time between MMAs.
+template <bool ACCUMULATE>
+__device__ __forceinline__ void umma_i8_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                           uint32_t desc_hi, uint32_t idesc)
+{
+    if constexpr (ACCUMULATE) {
+        asm volatile(
+            "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "setp.eq.b32 p, 0, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc));
+    } else {
+        asm volatile(
+            "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "setp.ne.b32 p, 0, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc));
+    }
+}
 // Arrive on `bar` once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
@@ -176,6 +200,15 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
 {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
            (1ull << 46) | (2ull << 61);
+}
+// The two 32-bit halves of that descriptor.
+__device__ __forceinline__ uint32_t smem_desc_sw128_lo(uint32_t saddr)
+{
+    return ((saddr & 0x3FFFFu) >> 4) | (1u << 16);
+}
+__host__ __device__ constexpr uint32_t smem_desc_sw128_hi()
+{
+    return (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
 }
 // Instruction descriptor for kind::i8, signed 8-bit A and B (both K-major), int32 D:
 //   [4,6) D format = 2 (s32), [7,10) A format = 1 (s8), [10,13) B format = 1 (s8),
