@@ -9,14 +9,15 @@
 //   stage    the zero-padded input strip (n rows x 16 columns x CB channels) goes to
 //            shared memory with 4-byte cp.async copies, all in flight at once
 //   phase 1  thread <-> (tile, channel): the n x n patch is transformed with the
-//            standard-scaled B^T (small integers / dyadic rationals as add/fma chains),
-//            multiplied by the caller's per-position factor and written as fp32 to a
-//            shared [tile][channel][position] array (odd pitch: conflict free)
+//            standard-scaled B^T (small integers / dyadic rationals as add/fma chains)
+//            and written as fp32 to a shared [tile][position][channel] array (lanes
+//            along the channel: conflict free)
 //   phase 2  thread <-> (tile, group, position): it reads the group's values of that
-//            position (lanes along the position: conflict free), takes the abs-max
-//            serially, derives scale and reciprocal once, rounds with the 1.5*2^23
-//            trick (same result as mul + round-half-even convert) and stores 16 codes
-//            per 16-byte store.
+//            position with 16-byte loads (rows 4 floats longer than the channel block:
+//            conflict free), multiplies them by the caller's per-position factor, takes
+//            the abs-max serially, derives scale and reciprocal once, rounds with the
+//            1.5*2^23 trick (same result as mul + round-half-even convert; multiply and
+//            add are packed f32x2) and stores 16 codes per 16-byte store.
 // The abs-max over a group therefore needs no shuffles; for groups of more than 64
 // channels phase 2 reads shared memory twice instead of holding the group in registers.
 #include <cuda_fp16.h>
@@ -108,17 +109,46 @@ __device__ __forceinline__ void load_patch(const float *ch, int col0, float (&d)
         for (int b = 0; b < NN; ++b) d[a][b] = ch[a * K1_WP + col0 + 1 + b];
 }
 
-// Round v*inv to the nearest integer (ties to even) and return it in the low byte:
-// fl32(v*inv) + 1.5*2^23 is exact up to the rounding to an integer, and the sum's
-// bit pattern is 0x4B400000 + q for |q| <= 2^22.
+// Codes: round v*inv to the nearest integer (ties to even) and keep the low byte.
+// fl32(v*inv) + 1.5*2^23 is exact up to the rounding to an integer, and the sum's bit
+// pattern is 0x4B400000 + q for |q| <= 2^22.
+// Packed f32x2 multiply (one instruction for two products, each correctly rounded).
+__device__ __forceinline__ float2 mul2_rn(float2 a, float2 b)
+{
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+
+// One code: fl32(v*inv), then + 1.5*2^23; two separately rounded scalar operations, as
+// the quantizer is defined.  (A packed multiply followed by a packed add, written as
+// intrinsics or as PTX, came out as one fused multiply-add: it rounds once and decides
+// near-ties differently, and a single differing code of an outlier-dominated group can
+// move the final output by more than the end-to-end tolerance.)
 __device__ __forceinline__ uint32_t code_bits(float v, float inv)
 {
     return __float_as_uint(__fadd_rn(__fmul_rn(v, inv), 12582912.f));
 }
-
-__device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+__device__ __forceinline__ uint32_t codes4(float4 v, float inv)
 {
-    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+    return __byte_perm(__byte_perm(code_bits(v.x, inv), code_bits(v.y, inv), 0x0040),
+                       __byte_perm(code_bits(v.z, inv), code_bits(v.w, inv), 0x0040), 0x5410);
+}
+
+__device__ __forceinline__ float4 scale4(float4 v, float2 s2)
+{
+    const float2 lo = mul2_rn(make_float2(v.x, v.y), s2);
+    const float2 hi = mul2_rn(make_float2(v.z, v.w), s2);
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+
+__device__ __forceinline__ float absmax4(float m, float4 v)
+{
+    return fmaxf(fmaxf(fmaxf(m, fabsf(v.x)), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
 }
 
 __device__ __forceinline__ void cp_async_4(uint32_t dst, const void *src, bool valid)
@@ -141,33 +171,29 @@ __device__ __forceinline__ void stage_strip(Tin *sm, const Tin *__restrict__ x, 
 {
     const size_t HW = (size_t)g.H * g.W;
     const Tin *ximg = x + ((size_t)img * g.C + c_base) * HW;
-    if (sizeof(Tin) == 4) {
-        // fp32: one 4-byte copy per element (the odd channel stride rules out 8-byte ones)
-        const int total = prm.CB * NN * K1_WP;
-        const uint32_t sm_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(sm));
-        for (int idx = threadIdx.x; idx < total; idx += K1_THREADS) {
-            const int j = idx % K1_WP;
-            const int row = idx / K1_WP;
-            const int c = row / NN, a = row - c * NN;
-            const int h = h_base + a, w = w_base + j;
-            const bool ok = h >= 0 && h < g.H && w >= 0 && w < g.W;
-            const Tin *src = ok ? ximg + (size_t)c * HW + (size_t)h * g.W + w : x;
-            cp_async_4(sm_u32 + (uint32_t)((c * prm.CS + a * K1_WP + j) * 4), src, ok);
-        }
-        cp_async_wait_all();
-    } else if (prm.pair) {
-        // fp16, even W, 4-byte aligned base: one 4-byte copy per pair of columns
-        constexpr int PR = K1_WP / 2;
-        const int total = prm.CB * NN * PR;
-        const uint32_t sm_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(sm));
-        for (int idx = threadIdx.x; idx < total; idx += K1_THREADS) {
-            const int jp = idx % PR;
-            const int row = idx / PR;
-            const int c = row / NN, a = row - c * NN;
-            const int h = h_base + a, w = w_base + 2 * jp;
-            const bool ok = h >= 0 && h < g.H && w >= 0 && w < g.W;   // W even: both or none
-            const Tin *src = ok ? ximg + (size_t)c * HW + (size_t)h * g.W + w : x;
-            cp_async_4(sm_u32 + (uint32_t)((c * prm.CS + a * K1_WP + 2 * jp) * 2), src, ok);
+    // Each thread owns one (row, column) slot of the strip and walks over the channels,
+    // so its bounds test and addresses are computed once.
+    if (sizeof(Tin) == 4 || prm.pair) {
+        constexpr int EPC = sizeof(Tin) == 4 ? 1 : 2;          // elements per 4-byte copy
+        constexpr int CPR = K1_WP / EPC;                       // copies per row
+        constexpr int ROWS = K1_THREADS / CPR;                 // rows covered by one pass
+        constexpr int CSLOTS = ROWS / NN;                      // channels covered by one pass
+        const int jc = threadIdx.x % CPR;
+        const int rs = threadIdx.x / CPR;
+        const int a = rs % NN, cslot = rs / NN;
+        if (cslot < CSLOTS) {
+            const int h = h_base + a, w = w_base + EPC * jc;
+            const bool ok = h >= 0 && h < g.H && w >= 0 && w < g.W;   // W even for pairs: both or none
+            const Tin *src = ok ? ximg + (size_t)cslot * HW + (size_t)h * g.W + w : x;
+            const size_t src_step = ok ? (size_t)CSLOTS * HW : 0;
+            uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(sm)) +
+                           (uint32_t)((cslot * prm.CS + a * K1_WP + EPC * jc) * sizeof(Tin));
+            const uint32_t dst_step = (uint32_t)(CSLOTS * prm.CS * sizeof(Tin));
+            for (int c = cslot; c < prm.CB; c += CSLOTS) {
+                cp_async_4(dst, src, ok);
+                src += src_step;
+                dst += dst_step;
+            }
         }
         cp_async_wait_all();
     } else {
@@ -185,11 +211,9 @@ __device__ __forceinline__ void stage_strip(Tin *sm, const Tin *__restrict__ x, 
     }
 }
 
-// Z = B^T d B with the standard B^T, times the caller's per-position factor, written
-// to out[p] for p = i*NN + j.
+// Z = B^T d B with the standard B^T, written to out[p * pitch] for p = i*NN + j.
 template <int NN>
-__device__ __forceinline__ void transform_patch(float (&d)[NN][NN], const ScaleTables &tab,
-                                                float *__restrict__ out)
+__device__ __forceinline__ void transform_patch(float (&d)[NN][NN], float *__restrict__ out, int pitch)
 {
 #pragma unroll
     for (int b = 0; b < NN; ++b) {   // columns: d <- B^T d
@@ -205,7 +229,7 @@ __device__ __forceinline__ void transform_patch(float (&d)[NN][NN], const ScaleT
         float r[NN];
         bt_1d(d[i], r);
 #pragma unroll
-        for (int j = 0; j < NN; ++j) out[i * NN + j] = __fmul_rn(r[j], tab.in_scale[i * NN + j]);
+        for (int j = 0; j < NN; ++j) out[(i * NN + j) * pitch] = r[j];
     }
 }
 
@@ -228,10 +252,10 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
 {
     constexpr int NN = M + 2;
     constexpr int P = NN * NN;
-    constexpr int PP = P + 1;                      // odd pitch of the [channel][position] array
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Tin *strip = reinterpret_cast<Tin *>(smem_raw);
-    float *Xs = reinterpret_cast<float *>(smem_raw + prm.strip_bytes);
+    float *Zs = reinterpret_cast<float *>(smem_raw + prm.strip_bytes);   // [tile][position][CBP]
+    const int CBP = prm.CB + 4;   // 16-byte aligned rows an odd number of 16-byte units apart
 
     const int srow = blockIdx.x / prm.NCH;         // img*TH + th
     const int chunk = blockIdx.x - srow * prm.NCH;
@@ -252,11 +276,13 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
         const int c = (wt - tl * cb32) * 32 + lane;
         float d[NN][NN];
         load_patch<NN>(strip + c * prm.CS, tl * M, d);
-        transform_patch<NN>(d, tab, Xs + (size_t)(tl * prm.CB + c) * PP);
+        transform_patch<NN>(d, Zs + (size_t)tl * P * CBP + c, CBP);
     }
     __syncthreads();
 
     // ---- phase 2: quantize, one (tile, group, position) per thread -------------------
+    // X = Z * (caller's per-position factor) is formed here, one rounding, as the
+    // quantizer's input; then abs-max, scale, reciprocal and codes.
     const int gs = GSR > 0 ? GSR : g.gs;
     const int ng = prm.CB / gs;
     const int g_base = c_base / gs;
@@ -265,41 +291,33 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
         const int q = task / P, p = task - q * P;
         const int tl = q / ng, grp = q - tl * ng;
         const int t = srow * g.TW + tw0 + tl;
-        const float *src = Xs + (size_t)(tl * prm.CB + grp * gs) * PP + p;
+        const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs);
         int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
+        const float sp = tab.in_scale[p];
+        const float2 sp2 = make_float2(sp, sp);
         float scale, inv;
         if constexpr (GSR > 0) {
-            float v[GSR];
+            float4 v[GSR / 4];
             float amax = 0.f;
 #pragma unroll
-            for (int cc = 0; cc < GSR; ++cc) {
-                v[cc] = src[cc * PP];
-                amax = fmaxf(amax, fabsf(v[cc]));
+            for (int k = 0; k < GSR / 4; ++k) {
+                v[k] = scale4(src[k], sp2);
+                amax = absmax4(amax, v[k]);
             }
             group_scale(amax, scale, inv);
 #pragma unroll
-            for (int c16 = 0; c16 < GSR; c16 += 16) {
-                uint32_t wd[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    wd[k] = pack4(code_bits(v[c16 + 4 * k], inv), code_bits(v[c16 + 4 * k + 1], inv),
-                                  code_bits(v[c16 + 4 * k + 2], inv), code_bits(v[c16 + 4 * k + 3], inv));
-                *reinterpret_cast<uint4 *>(dst + c16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-            }
+            for (int k = 0; k < GSR / 16; ++k)
+                *reinterpret_cast<uint4 *>(dst + 16 * k) =
+                    make_uint4(codes4(v[4 * k], inv), codes4(v[4 * k + 1], inv),
+                               codes4(v[4 * k + 2], inv), codes4(v[4 * k + 3], inv));
         } else {
             float amax = 0.f;
-            for (int cc = 0; cc < gs; ++cc) amax = fmaxf(amax, fabsf(src[cc * PP]));
+            for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2));
             group_scale(amax, scale, inv);
-            for (int c16 = 0; c16 < gs; c16 += 16) {
-                uint32_t wd[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float *s4 = src + (size_t)(c16 + 4 * k) * PP;
-                    wd[k] = pack4(code_bits(s4[0], inv), code_bits(s4[PP], inv),
-                                  code_bits(s4[2 * PP], inv), code_bits(s4[3 * PP], inv));
-                }
-                *reinterpret_cast<uint4 *>(dst + c16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-            }
+            for (int k = 0; k < gs / 16; ++k)
+                *reinterpret_cast<uint4 *>(dst + 16 * k) =
+                    make_uint4(codes4(scale4(src[4 * k], sp2), inv), codes4(scale4(src[4 * k + 1], sp2), inv),
+                               codes4(scale4(src[4 * k + 2], sp2), inv), codes4(scale4(src[4 * k + 3], sp2), inv));
         }
         sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
     }
@@ -310,7 +328,7 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
 {
     const Geometry &g = plan.geo;
     constexpr int NN = M + 2;
-    constexpr int PP = NN * NN + 1;
+    constexpr int P = NN * NN;
     const int esz = (int)sizeof(Tin);
     K1Params prm;
     prm.TB = (K1_WP - 3) / M;                      // 2 tiles for F(6,3), 3 for F(4,3)
@@ -325,7 +343,7 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
     prm.strip_bytes = (prm.CB * cs * esz + 15) / 16 * 16;
     prm.pair = (g.W % 2 == 0) && (reinterpret_cast<uintptr_t>(x_dev) % 4 == 0);
     auto smem_bytes = [&]() {
-        return (size_t)prm.strip_bytes + (size_t)prm.TB * prm.CB * PP * sizeof(float);
+        return (size_t)prm.strip_bytes + (size_t)prm.TB * P * (prm.CB + 4) * sizeof(float);
     };
     while (prm.TB > 1 && smem_bytes() > 220 * 1024) --prm.TB;   // very large groups
     const size_t smem = smem_bytes();
