@@ -143,12 +143,13 @@ class ClockSampler:
 
 # ---- CPU oracle legs -------------------------------------------------------------------
 
-def oracle_time_sample(layers, tensors, seconds, repeats=1):
+def oracle_time_sample(layers, tensors, seconds):
     """Times the oracle's forward pipeline on a sample of tiles of every layer.
 
-    Returns (ops, secs, description): direct-equivalent operations covered by the
-    sampled tiles and the CPU seconds they took (filter preparation excluded, as on
-    the GPU side).
+    Each layer gets an equal share of `seconds`: as many (randomly chosen) tiles as that
+    share allows, or, where the whole layer takes less, the whole layer several times.
+    Returns (ops, secs, description, threads): direct-equivalent operations covered and
+    the CPU seconds they took (filter preparation excluded, as on the GPU side).
     """
     import numpy as np
     from oracle import oracle as orc
@@ -159,22 +160,25 @@ def oracle_time_sample(layers, tensors, seconds, repeats=1):
         mats = orc.matrices(L.m, sB, sG)
         filt = orc.prepare_filters(w, L.m, L.gs, mats)
         rng = np.random.default_rng(L.seed + 7)
-        probe = min(T, 8)
-        tiles = np.sort(rng.choice(T, probe, replace=False))
-        t0 = time.perf_counter()
-        orc.wfq(x, w, L.m, L.gs, sB=sB, sG=sG, tiles=tiles, filters=filt)
-        dt = time.perf_counter() - t0
-        n = int(max(probe, min(T, per_layer / max(dt / probe, 1e-9))))
-        tiles = np.sort(rng.choice(T, n, replace=False))
-        best = None
-        for _ in range(repeats):
+
+        def run(n):
+            tiles = np.sort(rng.choice(T, n, replace=False))
             t0 = time.perf_counter()
             orc.wfq(x, w, L.m, L.gs, sB=sB, sG=sG, tiles=tiles, filters=filt)
-            dt = time.perf_counter() - t0
-            best = dt if best is None else min(best, dt)
-        total_ops += L.direct_ops * (n / T)
-        total_s += best
-        desc.append(f"{n}/{T}")
+            return time.perf_counter() - t0
+
+        n = min(T, 16)
+        dt = run(n)
+        while n < T and dt < 0.25 * per_layer:            # grow the sample towards the budget
+            n = min(T, max(2 * n, int(n * 0.8 * per_layer / max(dt, 1e-6))))
+            dt = run(n)
+        reps, spent = 1, dt
+        while n == T and spent + dt < per_layer:          # a small layer: whole layer, repeated
+            spent += run(n)
+            reps += 1
+        total_ops += L.direct_ops * (n / T) * reps
+        total_s += spent
+        desc.append(f"{n}/{T}" + (f"x{reps}" if reps > 1 else ""))
     return total_ops, total_s, "tiles per layer " + ",".join(desc), orc.num_threads()
 
 

@@ -41,7 +41,10 @@ __device__ __forceinline__ void at_1d(const float (&v)[M + 2], float (&o)[M])
     if constexpr (M == 4) at_f43(v, o); else at_f63(v, o);
 }
 
-template <int M>
+// STORE: 0 = element-wise with bounds checks (any W), 1 = 8-byte stores (W even),
+// 2 = 16-byte stores (F(4,3), W a multiple of 4).  With W a multiple of the store width
+// a tile row is either completely inside the image or completely outside.
+template <int M, int STORE>
 __global__ void __launch_bounds__(128)
 output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geometry g,
                         ScaleTables tab)
@@ -58,8 +61,14 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
 #pragma unroll
     for (int i = 0; i < NN; ++i)
 #pragma unroll
-        for (int j = 0; j < NN; ++j)
-            v[i][j] = __ldg(src + (size_t)(i * NN + j) * plane) * tab.out_scale[i * NN + j];
+        for (int j = 0; j < NN; ++j) {
+            v[i][j] = __ldg(src);
+            src += plane;
+        }
+#pragma unroll
+    for (int i = 0; i < NN; ++i)
+#pragma unroll
+        for (int j = 0; j < NN; ++j) v[i][j] *= tab.out_scale[i * NN + j];
 
     // columns: tmp[u][j] = sum_i VA[u][i] v[i][j]
     float tmp[M][NN];
@@ -74,20 +83,20 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
     }
 
     const int tw = t % g.TW;
-    const int th = (t / g.TW) % g.TH;
-    const int img = t / (g.TW * g.TH);
+    const int tq = t / g.TW;
+    const int th = tq % g.TH;
+    const int img = tq / g.TH;
     const int h0 = th * M, w0 = tw * M;
-    float *dst = y + (((size_t)img * g.K + k) * g.H + h0) * g.W + w0;
+    float *row = y + (((size_t)img * g.K + k) * g.H + h0) * g.W + w0;
     const bool full_w = (w0 + M <= g.W);
 #pragma unroll
     for (int u = 0; u < M; ++u) {
         float o[M];
         at_1d<M>(tmp[u], o);
         if (h0 + u < g.H) {
-            float *row = dst + (size_t)u * g.W;
-            if (full_w && (g.W % 4 == 0) && M == 4) {
+            if (STORE == 2 && full_w) {
                 *reinterpret_cast<float4 *>(row) = make_float4(o[0], o[1], o[2], o[3]);
-            } else if (full_w && (g.W % 2 == 0)) {
+            } else if (STORE >= 1 && full_w) {
 #pragma unroll
                 for (int v2 = 0; v2 < M; v2 += 2)
                     *reinterpret_cast<float2 *>(row + v2) = make_float2(o[v2], o[v2 + 1]);
@@ -97,6 +106,7 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
                     if (w0 + v2 < g.W) row[v2] = o[v2];
             }
         }
+        row += g.W;
     }
 }
 
@@ -116,8 +126,17 @@ cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStre
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     const float *Y = plan.ws.Y;
-    if (g.m == 4) return cudaLaunchKernelEx(&cfg, output_transform_kernel<4>, Y, y_dev, g, plan.tables);
-    return cudaLaunchKernelEx(&cfg, output_transform_kernel<6>, Y, y_dev, g, plan.tables);
+    // y_dev is 16-byte aligned; rows of an even W keep 8-byte alignment for every tile
+    if (g.m == 4) {
+        if (g.W % 4 == 0)
+            return cudaLaunchKernelEx(&cfg, output_transform_kernel<4, 2>, Y, y_dev, g, plan.tables);
+        if (g.W % 2 == 0)
+            return cudaLaunchKernelEx(&cfg, output_transform_kernel<4, 1>, Y, y_dev, g, plan.tables);
+        return cudaLaunchKernelEx(&cfg, output_transform_kernel<4, 0>, Y, y_dev, g, plan.tables);
+    }
+    if (g.W % 2 == 0)
+        return cudaLaunchKernelEx(&cfg, output_transform_kernel<6, 1>, Y, y_dev, g, plan.tables);
+    return cudaLaunchKernelEx(&cfg, output_transform_kernel<6, 0>, Y, y_dev, g, plan.tables);
 }
 
 }  // namespace wfq
