@@ -75,8 +75,8 @@ struct Cfg {
 
 // Bounded mbarrier wait.  Returns false (and records `where`) on timeout or when
 // another role of this CTA already gave up.  The loop body is the bare try_wait (which
-// suspends the thread in hardware for a while); clock and abort flag are looked at
-// every 1024 tries.
+// suspends the thread in hardware for up to a millisecond); clock and abort flag are
+// looked at every 64 tries.
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Shared *sh, int *status,
                                              int where)
 {
@@ -84,7 +84,7 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Shar
 #pragma unroll 1
     for (uint32_t it = 1;; ++it) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((it & 1023u) == 0) {
+        if ((it & 63u) == 0) {
             if (sh->abort) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
