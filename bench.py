@@ -37,6 +37,13 @@ UNIT = "TOPS"
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch (mean over the layers of a step)
+# from the ncu capture summarised in profiles/launches_cfg2_resnet18_stage.txt; cold-cache
+# reads, and output that is still dirty in L2 when the kernel ends is not counted.  Only the
+# default workload was captured; set an entry to None when its kernel changes.
+NCU_TRAFFIC_BYTES = {2: {"input_transform_quantize": 6.05e6, "gemm_dequantize": 13.6e6,
+                         "output_transform": 28.6e6}}
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -324,10 +331,14 @@ def run_wfq(args):
     else:
         peak, peak_src = FALLBACK_HBM_GBS, "fallback"
     achieved = tot_bytes[dom] / (tot_ms[dom] * 1e-3) / 1e9
+    traffic = None
+    if args.only_layer is None:
+        traffic = NCU_TRAFFIC_BYTES.get(args.config, {}).get(names[dom])
     roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                 "launches_per_step": len(layers),
                 "algorithmic_bytes_per_step": tot_bytes[dom],
+                "algorithmic_bytes_per_launch": tot_bytes[dom] / len(layers),
                 "all_kernels": {names[k]: {"us_per_step": tot_ms[k] * 1e3,
                                            "GBps": tot_bytes[k] / (tot_ms[k] * 1e-3) / 1e9,
                                            "frac": tot_bytes[k] / (tot_ms[k] * 1e-3) / 1e9 / peak}
