@@ -221,6 +221,25 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ---- aggregation over replicas ---------------------------------------------------------
+
+def max_over_ranks(value, device=None):
+    """The maximum of a per-rank time over all ranks (no-op without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(ops_per_replica, world, ms_per_step):
+    """Whole-job throughput in TOPS: every rank runs an independent replica of the
+    workload (the path needs no exchange), the job takes as long as its slowest rank."""
+    return world * ops_per_replica / (ms_per_step * 1e-3) / 1e12
+
+
 # ---- the CUDA path ---------------------------------------------------------------------
 
 def run_wfq(args):
@@ -292,12 +311,9 @@ def run_wfq(args):
     clocks = sampler.stop()
     ms_steps = [s.elapsed_time(e) for s, e in zip(starts, stops)]
     total_ms = float(sum(ms_steps))
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * step_ops / (ms_per_step * 1e-3) / 1e12
+    value = replica_throughput(step_ops, world, ms_per_step)
 
     # ---- per-kernel durations in the same chained order (events between the stages) ----
     names = ["input_transform_quantize", "gemm_dequantize", "output_transform"]
@@ -364,11 +380,8 @@ def run_wfq(args):
                 conv.forward_host(x, y)          # synchronous: copies + kernels + copy back
         torch.cuda.synchronize(dev)
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e = {"value": world * step_ops * esteps / dt / 1e12, "unit": UNIT,
+        dt = max_over_ranks(dt, dev)
+        e2e = {"value": replica_throughput(step_ops, world, dt * 1e3 / esteps), "unit": UNIT,
                "h2d_bytes_per_step": int(sum(x.numel() * x.element_size() for x in xh)),
                "d2h_bytes_per_step": int(sum(y.numel() * 4 for y in yh)), "steps": esteps}
 
