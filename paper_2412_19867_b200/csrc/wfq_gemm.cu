@@ -390,13 +390,15 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if constexpr (!DUMP) {
                 if (ok && active && row_ok) {
                     if constexpr (SWAP) {
-                        // row = output channel, columns = tiles: contiguous in Y[p][k][:]
+                        // row = output channel, columns = tiles: contiguous in Y[p][k][:];
+                        // 32-byte stores so that every instruction fills whole sectors
                         float *dst = a.Y + ((size_t)p * g.K + row) * g.Tp + col0;
 #pragma unroll
-                        for (int j4 = 0; j4 < CW / 4; ++j4)
-                            if (col0 + 4 * j4 + 3 < g.Tp)
-                                *reinterpret_cast<float4 *>(dst + 4 * j4) =
-                                    make_float4(acc[2 * j4].x, acc[2 * j4].y, acc[2 * j4 + 1].x, acc[2 * j4 + 1].y);
+                        for (int j8 = 0; j8 < CW / 8; ++j8)
+                            if (col0 + 8 * j8 + 7 < g.Tp)
+                                ptx::st_global_v8(dst + 8 * j8, acc[4 * j8].x, acc[4 * j8].y, acc[4 * j8 + 1].x,
+                                                  acc[4 * j8 + 1].y, acc[4 * j8 + 2].x, acc[4 * j8 + 2].y,
+                                                  acc[4 * j8 + 3].x, acc[4 * j8 + 3].y);
                     } else {
                         // row = tile: lanes write consecutive t of one Y[p][k][:] row
                         float *dst = a.Y + ((size_t)p * g.K + col0) * g.Tp + row;
@@ -473,7 +475,7 @@ void gemm_choose(const Geometry &g, bool *swap, int *bn)
     const long long normal = up(g.T, BM) * up(g.K, 64);
     const int bn_sw = g.T <= 32 ? 32 : 64;
     const long long swapped = up(g.K, BM) * up(g.T, bn_sw);
-    *swap = swapped < normal;
+    *swap = 5 * swapped < 4 * normal;   // swapped stores are less efficient: want >= 20 % less work
     *bn = *swap ? bn_sw : 64;
 }
 

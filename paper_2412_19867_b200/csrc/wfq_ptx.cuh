@@ -74,6 +74,15 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
         : "memory");
 }
 
+// 32-byte store (one full sector per lane); `p` must be 32-byte aligned.
+__device__ __forceinline__ void st_global_v8(float *p, float a, float b, float c, float d, float e,
+                                             float f, float g, float h)
+{
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d), "f"(e), "f"(f), "f"(g), "f"(h)
+                 : "memory");
+}
+
 // ---- programmatic dependent launch ---------------------------------------------------
 // Blocks until the grid this one was launched behind has completed and its writes are
 // visible (no-op for an ordinary launch).
