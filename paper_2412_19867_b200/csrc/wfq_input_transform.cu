@@ -4,8 +4,10 @@
 //   per (position, tile, channel group): amax -> scale, codes (Section 2 quantizer,
 //   one scale per group, dynamic abs-max)
 //
-// One CTA handles TB neighbouring tiles of one tile row and CB input channels (one or
-// two whole groups).  Three steps, separated by block barriers:
+// A work item is TB neighbouring tiles of one tile row and CB input channels (one or two
+// whole groups); persistent CTAs walk over the items.  Per item, separated by block
+// barriers (where shared memory allows it without costing a resident CTA, the next
+// item's strip is staged into a second buffer while this one is processed):
 //   stage    the zero-padded input strip (n rows x 16 columns x CB channels) goes to
 //            shared memory with 4-byte cp.async copies, all in flight at once
 //   phase 1  thread <-> (tile, channel): the n x n patch is transformed with the
@@ -31,12 +33,15 @@ constexpr int K1_THREADS = 128;
 constexpr int K1_WP = 16;        // staged columns per row (image columns w_base .. w_base+15)
 
 struct K1Params {
-    int TB;            // tiles per CTA
+    int TB;            // tiles per work item
     int NCH;           // chunks of TB tiles per tile row
-    int CB;            // channels per CTA (a multiple of the group size)
+    int NCB;           // channel blocks (C / CB)
+    int items;         // work items: N * TH * NCH * NCB
+    int CB;            // channels per work item (a multiple of the group size)
     int CS;            // shared-memory channel stride of the strip (elements)
     int strip_bytes;   // bytes of the strip, rounded up to 16
     int pair;          // 1: rows can be copied as aligned element pairs
+    int dbuf;          // 1: two strip buffers, the next item is staged during this one
 };
 
 // ---- 1-D input transforms with the standard B^T ------------------------------------
@@ -156,9 +161,14 @@ __device__ __forceinline__ void cp_async_4(uint32_t dst, const void *src, bool v
     const int n = valid ? 4 : 0;   // 0 source bytes: the destination is zero filled
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all()
+__device__ __forceinline__ void cp_async_commit()
 {
-    asm volatile("cp.async.wait_all;" ::: "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group()   // all but the N newest groups are done
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
 // ---- strip staging -----------------------------------------------------------------
@@ -195,18 +205,28 @@ __device__ __forceinline__ void stage_strip(Tin *sm, const Tin *__restrict__ x, 
                 dst += dst_step;
             }
         }
-        cp_async_wait_all();
     } else {
-        const int total = prm.CB * NN * K1_WP;
-        for (int idx = threadIdx.x; idx < total; idx += K1_THREADS) {
-            const int j = idx % K1_WP;
-            const int row = idx / K1_WP;
-            const int c = row / NN, a = row - c * NN;
+        // fp16 with an odd W or a 2-byte aligned base: plain 2-byte loads, eight channels
+        // in flight per thread (these copies are complete when the function returns)
+        constexpr int ROWS = K1_THREADS / K1_WP;               // 8 row slots per pass
+        constexpr int CSLOTS = ROWS / NN;                      // 1
+        const int j = threadIdx.x % K1_WP;
+        const int rs = threadIdx.x / K1_WP;
+        const int a = rs % NN, cslot = rs / NN;
+        if (cslot < CSLOTS) {
             const int h = h_base + a, w = w_base + j;
-            Tin v = Tin(0);
-            if (h >= 0 && h < g.H && w >= 0 && w < g.W)
-                v = __ldg(ximg + (size_t)c * HW + (size_t)h * g.W + w);
-            sm[c * prm.CS + a * K1_WP + j] = v;
+            const bool ok = h >= 0 && h < g.H && w >= 0 && w < g.W;
+            const Tin *src = ximg + (size_t)cslot * HW + (size_t)h * g.W + w;
+            Tin *dst = sm + cslot * prm.CS + a * K1_WP + j;
+            for (int c = cslot; c < prm.CB; c += 8 * CSLOTS) {     // CB is a multiple of 32
+                Tin v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = ok ? __ldg(src + (size_t)u * CSLOTS * HW) : Tin(0);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) dst[u * CSLOTS * prm.CS] = v[u];
+                src += (size_t)8 * CSLOTS * HW;
+                dst += 8 * CSLOTS * prm.CS;
+            }
         }
     }
 }
@@ -253,73 +273,100 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
     constexpr int NN = M + 2;
     constexpr int P = NN * NN;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    Tin *strip = reinterpret_cast<Tin *>(smem_raw);
-    float *Zs = reinterpret_cast<float *>(smem_raw + prm.strip_bytes);   // [tile][position][CBP]
+    // two strip buffers (the next item is staged while this one is transformed), then Z
+    float *Zs = reinterpret_cast<float *>(smem_raw + (1 + prm.dbuf) * prm.strip_bytes);   // [tile][position][CBP]
     const int CBP = prm.CB + 4;   // 16-byte aligned rows an odd number of 16-byte units apart
 
-    const int srow = blockIdx.x / prm.NCH;         // img*TH + th
-    const int chunk = blockIdx.x - srow * prm.NCH;
-    const int img = srow / g.TH, th = srow - img * g.TH;
-    const int tw0 = chunk * prm.TB;
-    const int ntile = min(prm.TB, g.TW - tw0);
-    const int c_base = blockIdx.y * prm.CB;
-
-    stage_strip<Tin, NN>(strip, x, g, prm, img, c_base, th * M - 1, tw0 * M - 2);
-    __syncthreads();
-
-    // ---- phase 1: transform, one (tile, channel) per thread --------------------------
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int NWARP = K1_THREADS / 32;
     const int cb32 = prm.CB >> 5;
-    for (int wt = warp; wt < ntile * cb32; wt += NWARP) {
-        const int tl = wt / cb32;
-        const int c = (wt - tl * cb32) * 32 + lane;
-        float d[NN][NN];
-        load_patch<NN>(strip + c * prm.CS, tl * M, d);
-        transform_patch<NN>(d, Zs + (size_t)tl * P * CBP + c, CBP);
-    }
-    __syncthreads();
-
-    // ---- phase 2: quantize, one (tile, group, position) per thread -------------------
-    // X = Z * (caller's per-position factor) is formed here, one rounding, as the
-    // quantizer's input; then abs-max, scale, reciprocal and codes.
     const int gs = GSR > 0 ? GSR : g.gs;
     const int ng = prm.CB / gs;
-    const int g_base = c_base / gs;
-    const int tasks = ntile * ng * P;
-    for (int task = threadIdx.x; task < tasks; task += K1_THREADS) {
-        const int q = task / P, p = task - q * P;
-        const int tl = q / ng, grp = q - tl * ng;
-        const int t = srow * g.TW + tw0 + tl;
-        const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs);
-        int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
-        const float sp = tab.in_scale[p];
-        const float2 sp2 = make_float2(sp, sp);
-        float scale, inv;
-        if constexpr (GSR > 0) {
-            float4 v[GSR / 4];
-            float amax = 0.f;
-#pragma unroll
-            for (int k = 0; k < GSR / 4; ++k) {
-                v[k] = scale4(src[k], sp2);
-                amax = absmax4(amax, v[k]);
-            }
-            group_scale(amax, scale, inv);
-#pragma unroll
-            for (int k = 0; k < GSR / 16; ++k)
-                *reinterpret_cast<uint4 *>(dst + 16 * k) =
-                    make_uint4(codes4(v[4 * k], inv), codes4(v[4 * k + 1], inv),
-                               codes4(v[4 * k + 2], inv), codes4(v[4 * k + 3], inv));
+
+    // item -> (tile row, chunk of tiles, channel block); channel blocks vary fastest so
+    // that CTAs running side by side read the same image rows
+    auto stage_item = [&](int item, int buf) {
+        const int cblk = item % prm.NCB, rest = item / prm.NCB;
+        const int srow = rest / prm.NCH, chunk = rest - srow * prm.NCH;
+        const int img = srow / g.TH, th = srow - img * g.TH;
+        stage_strip<Tin, NN>(reinterpret_cast<Tin *>(smem_raw + buf * prm.strip_bytes), x, g, prm, img,
+                             cblk * prm.CB, th * M - 1, chunk * prm.TB * M - 2);
+        cp_async_commit();
+    };
+
+    int item = blockIdx.x;
+    if (prm.dbuf && item < prm.items) stage_item(item, 0);
+    for (int it = 0; item < prm.items; ++it, item += gridDim.x) {
+        const int buf = prm.dbuf ? (it & 1) : 0;
+        const int next = item + gridDim.x;
+        if (!prm.dbuf) {
+            stage_item(item, 0);               // very large channel blocks: one buffer only
+            cp_async_wait_group<0>();
+        } else if (next < prm.items) {
+            stage_item(next, buf ^ 1);
+            cp_async_wait_group<1>();          // this item's copies have landed
         } else {
-            float amax = 0.f;
-            for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2));
-            group_scale(amax, scale, inv);
-            for (int k = 0; k < gs / 16; ++k)
-                *reinterpret_cast<uint4 *>(dst + 16 * k) =
-                    make_uint4(codes4(scale4(src[4 * k], sp2), inv), codes4(scale4(src[4 * k + 1], sp2), inv),
-                               codes4(scale4(src[4 * k + 2], sp2), inv), codes4(scale4(src[4 * k + 3], sp2), inv));
+            cp_async_wait_group<0>();
         }
-        sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
+        __syncthreads();
+
+        const Tin *strip = reinterpret_cast<const Tin *>(smem_raw + buf * prm.strip_bytes);
+        const int cblk = item % prm.NCB, rest = item / prm.NCB;
+        const int srow = rest / prm.NCH, chunk = rest - srow * prm.NCH;   // srow = img*TH + th
+        const int tw0 = chunk * prm.TB;
+        const int ntile = min(prm.TB, g.TW - tw0);
+        const int c_base = cblk * prm.CB;
+
+        // ---- phase 1: transform, one (tile, channel) per thread ----------------------
+        for (int wt = warp; wt < ntile * cb32; wt += NWARP) {
+            const int tl = wt / cb32;
+            const int c = (wt - tl * cb32) * 32 + lane;
+            float d[NN][NN];
+            load_patch<NN>(strip + c * prm.CS, tl * M, d);
+            transform_patch<NN>(d, Zs + (size_t)tl * P * CBP + c, CBP);
+        }
+        __syncthreads();
+
+        // ---- phase 2: quantize, one (tile, group, position) per thread -------------------
+        // X = Z * (caller's per-position factor) is formed here, one rounding, as the
+        // quantizer's input; then abs-max, scale, reciprocal and codes.
+        const int g_base = c_base / gs;
+        const int tasks = ntile * ng * P;
+        for (int task = threadIdx.x; task < tasks; task += K1_THREADS) {
+            const int q = task / P, p = task - q * P;
+            const int tl = q / ng, grp = q - tl * ng;
+            const int t = srow * g.TW + tw0 + tl;
+            const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs);
+            int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
+            const float sp = tab.in_scale[p];
+            const float2 sp2 = make_float2(sp, sp);
+            float scale, inv;
+            if constexpr (GSR > 0) {
+                float4 v[GSR / 4];
+                float amax = 0.f;
+    #pragma unroll
+                for (int k = 0; k < GSR / 4; ++k) {
+                    v[k] = scale4(src[k], sp2);
+                    amax = absmax4(amax, v[k]);
+                }
+                group_scale(amax, scale, inv);
+    #pragma unroll
+                for (int k = 0; k < GSR / 16; ++k)
+                    *reinterpret_cast<uint4 *>(dst + 16 * k) =
+                        make_uint4(codes4(v[4 * k], inv), codes4(v[4 * k + 1], inv),
+                                   codes4(v[4 * k + 2], inv), codes4(v[4 * k + 3], inv));
+            } else {
+                float amax = 0.f;
+                for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2));
+                group_scale(amax, scale, inv);
+                for (int k = 0; k < gs / 16; ++k)
+                    *reinterpret_cast<uint4 *>(dst + 16 * k) =
+                        make_uint4(codes4(scale4(src[4 * k], sp2), inv), codes4(scale4(src[4 * k + 1], sp2), inv),
+                                   codes4(scale4(src[4 * k + 2], sp2), inv), codes4(scale4(src[4 * k + 3], sp2), inv));
+            }
+            sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
+        }
+        __syncthreads();   // Z and this strip buffer are free again
     }
 }
 
@@ -343,9 +390,18 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
     prm.strip_bytes = (prm.CB * cs * esz + 15) / 16 * 16;
     prm.pair = (g.W % 2 == 0) && (reinterpret_cast<uintptr_t>(x_dev) % 4 == 0);
     auto smem_bytes = [&]() {
-        return (size_t)prm.strip_bytes + (size_t)prm.TB * P * (prm.CB + 4) * sizeof(float);
+        return (1 + prm.dbuf) * (size_t)prm.strip_bytes + (size_t)prm.TB * P * (prm.CB + 4) * sizeof(float);
     };
-    while (prm.TB > 1 && smem_bytes() > 220 * 1024) --prm.TB;   // very large groups
+    // Large groups get fewer tiles per item (aim: two or more CTAs per SM).  The second
+    // strip buffer is used only where it does not cost a resident CTA (registers allow four).
+    prm.dbuf = 0;
+    while (prm.TB > 1 && smem_bytes() > 113 * 1024) --prm.TB;
+    {
+        const size_t per_sm = 227 * 1024, one = smem_bytes() + 1024;
+        const size_t two = one + prm.strip_bytes;
+        const size_t n1 = per_sm / one < 4 ? per_sm / one : 4, n2 = per_sm / two < 4 ? per_sm / two : 4;
+        if (n2 >= 1 && n2 == n1) prm.dbuf = 1;
+    }
     const size_t smem = smem_bytes();
     prm.NCH = (g.TW + prm.TB - 1) / prm.TB;
 
@@ -354,7 +410,15 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    dim3 grid((unsigned)(g.N * g.TH * prm.NCH), (unsigned)(g.C / prm.CB));
+    prm.NCB = g.C / prm.CB;
+    prm.items = g.N * g.TH * prm.NCH * prm.NCB;
+    // persistent CTAs: as many as fit on the device at once
+    int per_sm = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, K1_THREADS, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorInvalidConfiguration;
+    const int resident = per_sm * plan.sm_count;
+    const int grid = prm.items < resident ? prm.items : resident;
     kern<<<grid, K1_THREADS, smem, stream>>>(static_cast<const Tin *>(x_dev), plan.ws.Xq, plan.ws.sX, g,
                                              plan.tables, prm);
     return cudaGetLastError();
