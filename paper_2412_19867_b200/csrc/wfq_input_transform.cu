@@ -18,8 +18,8 @@
 //            position with 16-byte loads (rows 4 floats longer than the channel block:
 //            conflict free), multiplies them by the caller's per-position factor, takes
 //            the abs-max serially, derives scale and reciprocal once, rounds with the
-//            1.5*2^23 trick (same result as mul + round-half-even convert; multiply and
-//            add are packed f32x2) and stores 16 codes per 16-byte store.
+//            1.5*2^23 trick (same result as mul + round-half-even convert; scalar multiply
+//            and add, each rounded) and stores 16 codes per 16-byte store.
 // The abs-max over a group therefore needs no shuffles; for groups of more than 64
 // channels phase 2 reads shared memory twice instead of holding the group in registers.
 #include <cuda_fp16.h>
