@@ -413,10 +413,10 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
     prm.NCB = g.C / prm.CB;
     prm.items = g.N * g.TH * prm.NCH * prm.NCB;
     // persistent CTAs: as many as fit on the device at once
-    int per_sm = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, K1_THREADS, smem);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                         (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    if (per_sm < 1) return cudaErrorInvalidConfiguration;
+    const int per_sm = resident_ctas_per_sm(kern, K1_THREADS, smem, 32);
     const int resident = per_sm * plan.sm_count;
     const int grid = prm.items < resident ? prm.items : resident;
     kern<<<grid, K1_THREADS, smem, stream>>>(static_cast<const Tin *>(x_dev), plan.ws.Xq, plan.ws.sX, g,

@@ -90,6 +90,26 @@ cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStre
 bool encode_tmap_bytes3d(CUtensorMap *map, const void *base, int inner, int rows, int planes,
                          int box_rows);
 
+
+// CTAs of `threads` threads and `smem` bytes of dynamic shared memory that fit on one SM of
+// this part (228 KB of shared memory with 1 KB reserved per CTA, 64 K registers allocated in
+// units of 256 per warp).  Used to size persistent grids; an overestimate only means that
+// some CTAs start later.
+template <typename Kernel>
+inline int resident_ctas_per_sm(Kernel kern, int threads, size_t smem, int cap)
+{
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return 1;
+    const int warps = (threads + 31) / 32;
+    const int regs_per_warp = (fa.numRegs * 32 + 255) / 256 * 256;
+    int n = 65536 / (regs_per_warp * warps);
+    const int by_smem = (int)((228 * 1024) / (smem + fa.sharedSizeBytes + 1024));
+    if (by_smem < n) n = by_smem;
+    if (2048 / threads < n) n = 2048 / threads;
+    if (cap < n) n = cap;
+    return n < 1 ? 1 : n;
+}
+
 int gemm_block_m();   // rows per unit of the contraction kernel (128)
 void gemm_choose(const Geometry &g, bool *swap, int *bn);
 
