@@ -11,7 +11,7 @@ by the time of the forward call (filter preparation is offline and not timed).
 
 One JSON line is printed by rank 0.  Besides the throughput it carries
   roofline      achieved HBM GB/s of the kernel that takes the most time in a step,
-                from CUDA events placed between the three stage calls
+                from CUDA events around the chain prefixes K1, K1+K2, K1+K2+K3
   e2e           the same metric through wfq_conv_forward_host (pinned host buffers,
                 host<->device copies inside the timed region)
   cpu_baseline  the CPU oracle timed on this machine's cores on a sample of tiles
@@ -315,27 +315,36 @@ def run_wfq(args):
     ms_per_step = total_ms / args.steps
     value = replica_throughput(step_ops, world, ms_per_step)
 
-    # ---- per-kernel durations in the same chained order (events between the stages) ----
+    # ---- per-kernel durations: differences of chain prefixes ---------------------------
+    # An event pair around a single short kernel adds several microseconds of launch
+    # latency to it.  So each layer is timed three times per step, as K1, K1+K2 and
+    # K1+K2+K3 (L2 flushed before each, one event pair around each prefix); the stage
+    # durations are the differences, the first one carries the pair's overhead.
     names = ["input_transform_quantize", "gemm_dequantize", "output_transform"]
     ksteps = min(args.steps, 100)
     kern_ms = [[0.0, 0.0, 0.0] for _ in layers]
     for _ in range(ksteps):
-        flush.zero_()
         evs = []
         for conv, x, y in zip(convs, xs, ys):
-            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-            e[0].record(stream)
-            b.wfq_input_transform_quantize(conv.plan, x.data_ptr(), sptr)
-            e[1].record(stream)
-            b.wfq_gemm_dequantize(conv.plan, sptr)
-            e[2].record(stream)
-            b.wfq_output_transform(conv.plan, y.data_ptr(), sptr)
-            e[3].record(stream)
-            evs.append(e)
+            per_prefix = []
+            for depth in (1, 2, 3):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                b.wfq_input_transform_quantize(conv.plan, x.data_ptr(), sptr)
+                if depth >= 2:
+                    b.wfq_gemm_dequantize(conv.plan, sptr)
+                if depth >= 3:
+                    b.wfq_output_transform(conv.plan, y.data_ptr(), sptr)
+                e1.record(stream)
+                per_prefix.append((e0, e1))
+            evs.append(per_prefix)
         torch.cuda.synchronize(dev)
-        for li, e in enumerate(evs):
-            for k in range(3):
-                kern_ms[li][k] += e[k].elapsed_time(e[k + 1]) / ksteps
+        for li, per_prefix in enumerate(evs):
+            t = [a.elapsed_time(z) for a, z in per_prefix]
+            kern_ms[li][0] += t[0] / ksteps
+            kern_ms[li][1] += (t[1] - t[0]) / ksteps
+            kern_ms[li][2] += (t[2] - t[1]) / ksteps
     abytes = [algorithmic_bytes(L) for L in layers]
     tot_ms = [sum(kern_ms[li][k] for li in range(len(layers))) for k in range(3)]
     tot_bytes = [sum(abytes[li][names[k]] for li in range(len(layers))) for k in range(3)]
