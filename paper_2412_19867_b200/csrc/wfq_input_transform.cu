@@ -19,7 +19,7 @@
 //            conflict free), multiplies them by the caller's per-position factor, takes
 //            the abs-max serially, derives scale and reciprocal once, rounds with the
 //            1.5*2^23 trick (same result as mul + round-half-even convert; scalar multiply
-//            and add, each rounded) and stores 16 codes per 16-byte store.
+//            and add, each rounded) and stores 32 codes per 32-byte store.
 // The abs-max over a group therefore needs no shuffles; for groups of more than 64
 // channels phase 2 reads shared memory twice instead of holding the group in registers.
 #include <cuda_fp16.h>
@@ -154,6 +154,15 @@ __device__ __forceinline__ float4 scale4(float4 v, float2 s2)
 __device__ __forceinline__ float absmax4(float m, float4 v)
 {
     return fmaxf(fmaxf(fmaxf(m, fabsf(v.x)), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+}
+
+// 32-byte store (one full sector); `p` must be 32-byte aligned.
+__device__ __forceinline__ void st_global_v8_b32(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
+                                                 uint32_t e, uint32_t f, uint32_t g, uint32_t h)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d), "r"(e), "r"(f), "r"(g), "r"(h)
+                 : "memory");
 }
 
 __device__ __forceinline__ void cp_async_4(uint32_t dst, const void *src, bool valid)
@@ -351,18 +360,21 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
                 }
                 group_scale(amax, scale, inv);
     #pragma unroll
-                for (int k = 0; k < GSR / 16; ++k)
-                    *reinterpret_cast<uint4 *>(dst + 16 * k) =
-                        make_uint4(codes4(v[4 * k], inv), codes4(v[4 * k + 1], inv),
-                                   codes4(v[4 * k + 2], inv), codes4(v[4 * k + 3], inv));
+                for (int k = 0; k < GSR / 32; ++k)        // 32 codes = one full sector per store
+                    st_global_v8_b32(dst + 32 * k, codes4(v[8 * k], inv), codes4(v[8 * k + 1], inv),
+                                     codes4(v[8 * k + 2], inv), codes4(v[8 * k + 3], inv),
+                                     codes4(v[8 * k + 4], inv), codes4(v[8 * k + 5], inv),
+                                     codes4(v[8 * k + 6], inv), codes4(v[8 * k + 7], inv));
             } else {
                 float amax = 0.f;
                 for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2));
                 group_scale(amax, scale, inv);
-                for (int k = 0; k < gs / 16; ++k)
-                    *reinterpret_cast<uint4 *>(dst + 16 * k) =
-                        make_uint4(codes4(scale4(src[4 * k], sp2), inv), codes4(scale4(src[4 * k + 1], sp2), inv),
-                                   codes4(scale4(src[4 * k + 2], sp2), inv), codes4(scale4(src[4 * k + 3], sp2), inv));
+                for (int k = 0; k < gs / 32; ++k)
+                    st_global_v8_b32(dst + 32 * k, codes4(scale4(src[8 * k], sp2), inv),
+                                     codes4(scale4(src[8 * k + 1], sp2), inv), codes4(scale4(src[8 * k + 2], sp2), inv),
+                                     codes4(scale4(src[8 * k + 3], sp2), inv), codes4(scale4(src[8 * k + 4], sp2), inv),
+                                     codes4(scale4(src[8 * k + 5], sp2), inv), codes4(scale4(src[8 * k + 6], sp2), inv),
+                                     codes4(scale4(src[8 * k + 7], sp2), inv));
             }
             sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
         }
