@@ -74,11 +74,12 @@ struct Cfg {
 };
 
 // Bounded mbarrier wait.  Returns false (and records `where`) on timeout or when
-// another role of this CTA already gave up.  The loop body is the bare try_wait (which
-// suspends the thread in hardware for up to a millisecond); clock and abort flag are
-// looked at every 64 tries.
-__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Shared *sh, int *status,
-                                             int where)
+// another role of this CTA already gave up.  The common case, a phase that has already
+// completed, is one try_wait inline; the waiting loop is kept out of line so that the
+// role loops stay short (their instructions sit on the critical path between MMAs).
+// In the loop the bare try_wait suspends the thread in hardware for up to a
+// millisecond; clock and abort flag are looked at every 64 tries.
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, Shared *sh, int *status, int where)
 {
     long long t0 = 0;
 #pragma unroll 1
@@ -100,6 +101,12 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Shar
         }
     }
 }
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Shared *sh, int *status,
+                                             int where)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    return wait_slow(bar, parity, sh, status, where);
+}
 
 // Bounded wait for copies that may still be in flight when a role gives up.
 __device__ __forceinline__ void drain(uint32_t bar, uint32_t parity)
@@ -118,6 +125,74 @@ struct GemmArgs {
     int32_t *acc_dump;        // [P][T][K][G] or null
     int *status;
 };
+
+// MMA issue loop for the common shapes in which the chunks tile a stage exactly
+// (GSTEPS MMAs per group, CGT groups per chunk, GSTEPS * CGT in {2, 4} MMAs per chunk):
+// per chunk one slot wait, the chunk's MMAs as straight-line code with constant
+// descriptor offsets and accumulate flags, one commit.  The generic loop in the kernel
+// spends several hundred cycles per MMA on its bookkeeping, which made the issuing
+// warp the bottleneck of every layer with more than one chunk per unit.
+template <int BN, int GSTEPS, int CGT>
+__device__ __forceinline__ void mma_issue_aligned(Shared *sh, uint32_t tiles_lo, uint32_t tmem_base,
+                                                  int units, int KB, int last_slices, int lane,
+                                                  int *status)
+{
+    using C = Cfg<BN>;
+    constexpr int CHUNK_STEPS = GSTEPS * CGT;            // MMAs per chunk
+    constexpr int NCH = (BK / UK) / CHUNK_STEPS;         // chunks per stage
+    static_assert(NCH >= 1 && NCH * CHUNK_STEPS == BK / UK, "chunks must tile a stage");
+    constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
+    constexpr uint32_t dhi = ptx::smem_desc_sw128_hi();
+    const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
+    const uint32_t acc0 = ptx::smem_u32(&sh->acc_full[0]), free0 = ptx::smem_u32(&sh->slot_free[0]);
+    int stage = 0, slot = 0;
+    uint32_t phase = 0, sphase = 0;
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+        for (int kb = 0; kb < KB; ++kb) {
+            const int nslice = kb == KB - 1 ? last_slices : BK / UK;
+            if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8u * stage, phase, sh, status, kWaitSmemFull)))
+                return;
+            const uint32_t a_lo = tiles_lo + (uint32_t)(stage * (C::STAGE_BYTES >> 4));
+            const uint32_t b_lo = a_lo + (uint32_t)(A_BYTES >> 4);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                if (c * CHUNK_STEPS < nslice) {           // the chunk has at least one group
+                    if (!__all_sync(0xffffffffu, wait_bounded(free0 + 8u * slot, sphase ^ 1u, sh, status,
+                                                              kWaitTmemEmpty)))
+                        return;
+                    ptx::tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t d = tmem_base + (uint32_t)(slot * SLOT_COLS);
+                        if ((c + 1) * CHUNK_STEPS <= nslice) {
+#pragma unroll
+                            for (int s = 0; s < CHUNK_STEPS; ++s) {
+                                const uint32_t off = 2u * (uint32_t)(c * CHUNK_STEPS + s);
+                                if (s % GSTEPS) ptx::umma_i8_lo<true>(d + (s / GSTEPS) * BN, a_lo + off, b_lo + off, dhi, idesc);
+                                else ptx::umma_i8_lo<false>(d + (s / GSTEPS) * BN, a_lo + off, b_lo + off, dhi, idesc);
+                            }
+                        } else {
+                            // last stage of a unit whose channel count is not a multiple of 128
+#pragma unroll
+                            for (int s = 0; s < CHUNK_STEPS; ++s) {
+                                const uint32_t off = 2u * (uint32_t)(c * CHUNK_STEPS + s);
+                                if (c * CHUNK_STEPS + s < nslice) {
+                                    if (s % GSTEPS) ptx::umma_i8_lo<true>(d + (s / GSTEPS) * BN, a_lo + off, b_lo + off, dhi, idesc);
+                                    else ptx::umma_i8_lo<false>(d + (s / GSTEPS) * BN, a_lo + off, b_lo + off, dhi, idesc);
+                                }
+                            }
+                        }
+                        ptx::umma_commit(acc0 + 8u * slot);
+                    }
+                    __syncwarp();
+                    if (++slot == NSLOT) { slot = 0; sphase ^= 1u; }
+                }
+            }
+            if (lane == 0) ptx::umma_commit(empty0 + 8u * stage);
+            __syncwarp();
+            if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
+        }
+    }
+}
 
 template <int BN, bool SWAP, bool DUMP>
 __global__ void __launch_bounds__(NUM_THREADS, 2)
@@ -217,9 +292,22 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         constexpr uint32_t dhi = ptx::smem_desc_sw128_hi();
         const uint32_t tiles_lo = ptx::smem_desc_sw128_lo(ptx::smem_u32(tiles));
         const int chunk_steps = cg * gs_steps;       // MMAs per full chunk
+        const int last_slices = (g.C - (KB - 1) * BK) / UK;
         int stage = 0, slot = 0;
         uint32_t phase = 0, sphase = 0;
         bool ok = true;
+        // shapes whose chunks tile a stage exactly take the straight-line issue loop
+        if (gs_steps == 2 && cg == 2) {
+            mma_issue_aligned<BN, 2, 2>(sh, tiles_lo, tmem_base, units, KB, last_slices, lane, status);
+            ok = false;
+        } else if (gs_steps == 4 && cg == 1) {
+            mma_issue_aligned<BN, 4, 1>(sh, tiles_lo, tmem_base, units, KB, last_slices, lane, status);
+            ok = false;
+        } else if (gs_steps == 1 && cg == C::CG_MAX && C::CG_MAX <= 4) {
+            mma_issue_aligned<BN, 1, (C::CG_MAX <= 4 ? C::CG_MAX : 4)>(sh, tiles_lo, tmem_base, units, KB,
+                                                                    last_slices, lane, status);
+            ok = false;
+        }
         for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
             int step = 0;          // MMA step within the chunk
             int in_group = 0;      // MMA step within the group
