@@ -83,6 +83,41 @@ __device__ __forceinline__ void bt_1d(const float (&d)[8], float (&r)[8])
     r[6] = f - g;
 }
 
+// The same two transforms on two columns at once (packed f32x2 arithmetic: one
+// instruction per pair, each component rounded as in the scalar form).
+__device__ __forceinline__ float2 f2(float v) { return make_float2(v, v); }
+
+__device__ __forceinline__ void bt_1d(const float2 (&d)[6], float2 (&r)[6])
+{
+    r[0] = __ffma2_rn(f2(4.f), d[0], __ffma2_rn(f2(-5.f), d[2], d[4]));
+    const float2 a = __ffma2_rn(f2(-4.f), d[2], d[4]);
+    const float2 b = __ffma2_rn(f2(-4.f), d[1], d[3]);
+    r[1] = __fadd2_rn(a, b);
+    r[2] = __ffma2_rn(f2(-1.f), b, a);
+    const float2 c = __ffma2_rn(f2(-1.f), d[2], d[4]);
+    const float2 t = __ffma2_rn(f2(-1.f), d[1], d[3]);
+    r[3] = __ffma2_rn(f2(2.f), t, c);
+    r[4] = __ffma2_rn(f2(-2.f), t, c);
+    r[5] = __ffma2_rn(f2(4.f), d[1], __ffma2_rn(f2(-5.f), d[3], d[5]));
+}
+
+__device__ __forceinline__ void bt_1d(const float2 (&d)[8], float2 (&r)[8])
+{
+    r[0] = __ffma2_rn(f2(5.25f), __ffma2_rn(f2(-1.f), d[2], d[4]), __ffma2_rn(f2(-1.f), d[6], d[0]));
+    r[7] = __ffma2_rn(f2(5.25f), __ffma2_rn(f2(-1.f), d[5], d[3]), __ffma2_rn(f2(-1.f), d[1], d[7]));
+    const float2 a = __ffma2_rn(f2(-4.25f), d[4], __fadd2_rn(d[2], d[6]));
+    const float2 b = __ffma2_rn(f2(-4.25f), d[3], __fadd2_rn(d[1], d[5]));
+    r[1] = __fadd2_rn(a, b);
+    r[2] = __ffma2_rn(f2(-1.f), b, a);
+    const float2 c = __ffma2_rn(f2(-1.25f), d[4], __ffma2_rn(f2(0.25f), d[2], d[6]));
+    const float2 e = __ffma2_rn(f2(2.f), d[5], __ffma2_rn(f2(-2.5f), d[3], __fmul2_rn(f2(0.5f), d[1])));
+    r[3] = __fadd2_rn(c, e);
+    r[4] = __ffma2_rn(f2(-1.f), e, c);
+    const float2 f = __ffma2_rn(f2(-5.f), d[4], __ffma2_rn(f2(4.f), d[2], d[6]));
+    const float2 g = __ffma2_rn(f2(0.5f), d[5], __ffma2_rn(f2(-2.5f), d[3], __fmul2_rn(f2(2.f), d[1])));
+    r[5] = __fadd2_rn(f, g);
+    r[6] = __ffma2_rn(f2(-1.f), g, f);
+}
 
 // ---- patch load from the staged strip ---------------------------------------------
 // `ch` points at the channel's plane in smem; `col0` is the (even) smem column whose
@@ -245,13 +280,16 @@ template <int NN>
 __device__ __forceinline__ void transform_patch(float (&d)[NN][NN], float *__restrict__ out, int pitch)
 {
 #pragma unroll
-    for (int b = 0; b < NN; ++b) {   // columns: d <- B^T d
-        float col[NN], r[NN];
+    for (int b = 0; b < NN; b += 2) {   // columns, two at a time: d <- B^T d
+        float2 col[NN], r[NN];
 #pragma unroll
-        for (int a = 0; a < NN; ++a) col[a] = d[a][b];
+        for (int a = 0; a < NN; ++a) col[a] = make_float2(d[a][b], d[a][b + 1]);
         bt_1d(col, r);
 #pragma unroll
-        for (int a = 0; a < NN; ++a) d[a][b] = r[a];
+        for (int a = 0; a < NN; ++a) {
+            d[a][b] = r[a].x;
+            d[a][b + 1] = r[a].y;
+        }
     }
 #pragma unroll
     for (int i = 0; i < NN; ++i) {   // rows: Z[i][:] = (B^T d)[i][:] B
