@@ -45,6 +45,10 @@ SMALL = [
     Layer(1, 256, 64, 20, 20, 4, 256, "f32", "gauss_outlier", "gauss_chan", 1, 0, 2),   # gs=256, fp32
     Layer(2, 32, 40, 9, 11, 4, 32, "f32", "gauss_outlier", "gauss_chan", 1, 0, 3),      # odd W, K=40
     Layer(1, 96, 32, 13, 13, 6, 96, "f16", "silu_outlier", "kaiming_chan", 4, 0, 4),    # gs=96
+    # few tiles, many output channels, groups of 32: output channels on the accumulator rows,
+    # four groups per chunk; with whole 128-channel stages and with a 32-channel last stage
+    Layer(1, 128, 128, 8, 8, 4, 32, "f16", "silu_outlier", "kaiming_chan", 4, 0, 5),
+    Layer(2, 160, 192, 8, 8, 4, 32, "f16", "silu_outlier", "kaiming_chan", 4, 0, 6),
 ]
 
 
