@@ -56,6 +56,8 @@ def parse_args():
                     help="restrict the workload to one layer of the configuration (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="enqueue every step with stream launches instead of replaying a CUDA graph")
     ap.add_argument("--cpu-seconds", type=float, default=16.0,
                     help="CPU time budget of the oracle baseline")
     return ap.parse_args()
@@ -278,9 +280,34 @@ def run_wfq(args):
     step_ops = float(sum(L.direct_ops for L in layers))
     sptr = stream.cuda_stream
 
-    def step():
+    def enqueue(stream_ptr):
         for conv, x, y in zip(convs, xs, ys):
-            b.wfq_conv_forward(conv.plan, x.data_ptr(), y.data_ptr(), sptr)
+            b.wfq_conv_forward(conv.plan, x.data_ptr(), y.data_ptr(), stream_ptr)
+
+    # One step = the forward calls of all layers.  They are captured once into a CUDA graph
+    # and replayed (same kernels, same order, one submission per step); stream launches are
+    # the fallback and what --no-graph selects.
+    enqueue(sptr)
+    torch.cuda.synchronize(dev)
+    graph, launch_mode = None, "stream launches"
+    if not args.no_graph:
+        try:
+            side = torch.cuda.Stream(dev)
+            side.wait_stream(stream)
+            cand = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(cand, stream=side):
+                enqueue(side.cuda_stream)
+            torch.cuda.synchronize(dev)
+            graph, launch_mode = cand, "CUDA graph replay"
+        except Exception as exc:   # capture is an optimisation of the submission only
+            print(f"bench: graph capture failed ({exc!r}); using stream launches", file=sys.stderr)
+            torch.cuda.synchronize(dev)
+
+    def step():
+        if graph is not None:
+            graph.replay()
+        else:
+            enqueue(sptr)
 
     def barrier():
         if world > 1:
@@ -437,7 +464,7 @@ def run_wfq(args):
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
                 "config": {"workload": workload_name(args.config) +
                            ("" if args.only_layer is None else f" (layer {args.only_layer} only)"),
-                           "layers": len(layers),
+                           "layers": len(layers), "launch": launch_mode,
                            "l2": "flushed before every step (256 MiB memset outside the step's "
                                  "event pair)",
                            "parallelism": "replicas" if world > 1 else "single GPU"},
