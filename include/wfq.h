@@ -171,9 +171,13 @@ wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev,
 
 /*
  * Same computation with HOST buffers: copies x to the device, runs the three kernels,
- * copies y back, all on `stream`, then waits for the stream (synchronous).  The plan
- * allocates device staging for x and y on first use.  x_host/y_host should be pinned
- * for full copy speed.
+ * copies y back, then waits for `stream` (synchronous).  The plan allocates device
+ * staging for x and y on first use.  x_host/y_host should be pinned for full copy speed.
+ * Batches of three or more images with more than 12 MB to move are cut into chunks of
+ * whole images that alternate between two streams owned by the plan (created on first
+ * use, ordered after the work already on `stream`, and `stream` waits for them), so that
+ * copies in, kernels and copies out overlap; the results are identical to the unchunked
+ * path.
  */
 wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *y_host,
                                    void *stream);

@@ -266,6 +266,56 @@ wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev,
     return cuda_status(e);
 }
 
+// Number of chunks for the pipelined host path: a divisor of N (whole images per chunk,
+// all chunks alike), at least three so that two chunks fit the caller's workspace, and
+// only for transfers large enough to pay for the extra launches.
+static int pick_host_chunks(const wfq_plan *plan, size_t xb, size_t yb)
+{
+    const int N = plan->geo.N;
+    if (N < 3 || xb + yb < ((size_t)12 << 20)) return 1;
+    const int prefer[] = {4, 3, 5, 6, 7, 8};
+    for (int c : prefer)
+        if (N % c == 0 && (xb / c) % 16 == 0 && (yb / c) % 16 == 0) return c;   // aligned chunk starts
+    return 1;
+}
+
+// (Re)builds the two chunk plans from the parent's current state.  Cheap: no device work
+// except, the first time, the creation of two streams and three events.
+static wfq_status_t setup_host_pipeline(wfq_plan *plan)
+{
+    const wfq::Geometry &g = plan->geo;
+    const int nc = g.N / plan->host_chunks;
+    for (int s = 0; s < 2; ++s) {
+        if (!plan->sub[s]) {
+            wfq_status_t st = wfq_plan_create(&plan->sub[s], nc, g.C, g.K, g.H, g.W, g.m, 3, g.gs, 8);
+            if (st != WFQ_OK) return st;
+            plan->sub[s]->borrowed = true;
+        }
+        wfq_plan *q = plan->sub[s];
+        q->in_dtype = plan->in_dtype;
+        // same orientation of the contraction as the whole batch: identical arithmetic
+        q->gemm_swap = plan->gemm_swap;
+        q->gemm_bn = plan->gemm_bn;
+        const size_t slice = align_up(q->ws.total, 1024);
+        if (2 * slice > plan->ws.total) return WFQ_ERR_UNSUPPORTED;
+        wfq_status_t st = wfq_plan_set_workspace(q, reinterpret_cast<char *>(plan->ws.Xq) + s * slice, slice);
+        if (st != WFQ_OK) return st;
+        q->Wq = plan->Wq; q->sW = plan->sW; q->status = plan->status;
+        q->tables = plan->tables;
+        q->tmap_wq = plan->tmap_wq; q->tmap_wq_ok = plan->tmap_wq_ok;
+        q->device = plan->device; q->sm_count = plan->sm_count;
+        q->prepared = true;
+        if (!plan->host_stream[s] &&
+            cudaStreamCreateWithFlags(&plan->host_stream[s], cudaStreamNonBlocking) != cudaSuccess)
+            return WFQ_ERR_CUDA;
+    }
+    for (int i = 0; i < 3; ++i)
+        if (!plan->host_event[i] &&
+            cudaEventCreateWithFlags(&plan->host_event[i], cudaEventDisableTiming) != cudaSuccess)
+            return WFQ_ERR_CUDA;
+    return WFQ_OK;
+}
+
 wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *y_host,
                                    void *stream)
 {
@@ -280,6 +330,40 @@ wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *
         return cuda_status(e);
     if (!plan->y_stage && (e = cudaMalloc(&plan->y_stage, yb)) != cudaSuccess) return cuda_status(e);
     cudaStream_t st = as_stream(stream);
+
+    if (plan->host_chunks == 0) plan->host_chunks = pick_host_chunks(plan, xb, yb);
+    if (plan->host_chunks > 1 && setup_host_pipeline(plan) != WFQ_OK) plan->host_chunks = 1;
+
+    if (plan->host_chunks > 1) {
+        const int chunks = plan->host_chunks;
+        const size_t xc = xb / chunks, yc = yb / chunks;
+        // the internal streams start after the work already queued on the caller's stream
+        if (cudaEventRecord(plan->host_event[2], st) != cudaSuccess) return WFQ_ERR_CUDA;
+        for (int i = 0; i < 2; ++i)
+            if (cudaStreamWaitEvent(plan->host_stream[i], plan->host_event[2], 0) != cudaSuccess)
+                return WFQ_ERR_CUDA;
+        for (int c = 0; c < chunks; ++c) {
+            cudaStream_t cs = plan->host_stream[c & 1];
+            char *xd = static_cast<char *>(plan->x_stage) + (size_t)c * xc;
+            float *yd = plan->y_stage + (size_t)c * (yc / sizeof(float));
+            if (cudaMemcpyAsync(xd, static_cast<const char *>(x_host) + (size_t)c * xc, xc,
+                                cudaMemcpyHostToDevice, cs) != cudaSuccess)
+                return WFQ_ERR_CUDA;
+            s = wfq_conv_forward(plan->sub[c & 1], xd, yd, cs);
+            if (s != WFQ_OK) return s;
+            if (cudaMemcpyAsync(reinterpret_cast<char *>(y_host) + (size_t)c * yc, yd, yc,
+                                cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+                return WFQ_ERR_CUDA;
+        }
+        // and the caller's stream continues after both of them
+        for (int i = 0; i < 2; ++i) {
+            if (cudaEventRecord(plan->host_event[i], plan->host_stream[i]) != cudaSuccess ||
+                cudaStreamWaitEvent(st, plan->host_event[i], 0) != cudaSuccess)
+                return WFQ_ERR_CUDA;
+        }
+        return cuda_status(cudaStreamSynchronize(st));
+    }
+
     if ((e = cudaMemcpyAsync(plan->x_stage, x_host, xb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
         return WFQ_ERR_CUDA;
     s = wfq_conv_forward(plan, plan->x_stage, plan->y_stage, stream);
@@ -334,6 +418,13 @@ wfq_status_t wfq_check_device_status(wfq_plan_t *plan, void *stream, int *where)
 wfq_status_t wfq_plan_destroy(wfq_plan_t *plan)
 {
     if (!plan) return WFQ_OK;
+    for (int i = 0; i < 2; ++i) {
+        if (plan->sub[i]) delete plan->sub[i];       // borrowed device memory: nothing to free
+        if (plan->host_stream[i]) cudaStreamDestroy(plan->host_stream[i]);
+    }
+    for (int i = 0; i < 3; ++i)
+        if (plan->host_event[i]) cudaEventDestroy(plan->host_event[i]);
+    if (plan->borrowed) { delete plan; return WFQ_OK; }
     if (plan->Wq) cudaFree(plan->Wq);
     if (plan->sW) cudaFree(plan->sW);
     if (plan->status) cudaFree(plan->status);

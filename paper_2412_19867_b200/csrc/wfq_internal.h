@@ -73,6 +73,17 @@ struct wfq_plan {
     bool tmap_xq_ok = false, tmap_wq_ok = false;
     bool gemm_swap = false;    // contraction rows are output channels instead of tiles
     int gemm_bn = 64;          // columns per unit of the contraction
+
+    // wfq_conv_forward_host on batches of several images: the batch is cut into chunks
+    // of whole images that alternate between two internal streams, so that the copy in
+    // of one chunk, the kernels of another and the copy out of a third overlap.  The two
+    // sub-plans describe one chunk each; they borrow this plan's filters, scale tables,
+    // status word and halves of its workspace.
+    wfq_plan *sub[2] = {nullptr, nullptr};
+    int host_chunks = 0;                     // 0: not decided yet, 1: no chunking
+    cudaStream_t host_stream[2] = {nullptr, nullptr};
+    cudaEvent_t host_event[3] = {nullptr, nullptr, nullptr};
+    bool borrowed = false;                   // this is a sub-plan: it owns no device memory
 };
 
 namespace wfq {

@@ -100,6 +100,24 @@ def test_host_buffer_entry_point_matches_device_one():
     conv.close()
 
 
+def test_host_buffer_entry_point_in_chunks_matches_device_one():
+    """A batch large enough for the pipelined host path (chunks of whole images on two
+    internal streams): same bits as the device entry point, twice in a row."""
+    import torch
+    from tests.gpu_util import make_conv
+    L = Layer(8, 64, 128, 56, 56, 6, 64, "f16", "relu_heavy", "kaiming", 2, 0, 7)
+    conv, (x, w, sB, sG) = make_conv(L)
+    xd = torch.from_numpy(x).cuda()
+    y_dev = conv.forward(xd).cpu()
+    xh = torch.from_numpy(x).pin_memory()
+    for _ in range(2):
+        yh = torch.zeros(y_dev.shape, dtype=torch.float32).pin_memory()
+        conv.forward_host(xh, yh)
+        assert torch.equal(yh, y_dev)
+    conv.check_status()
+    conv.close()
+
+
 def test_misaligned_or_null_device_pointers_are_rejected():
     import torch
     from paper_2412_19867_b200 import binding as b
