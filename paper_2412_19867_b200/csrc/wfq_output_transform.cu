@@ -41,72 +41,116 @@ __device__ __forceinline__ void at_1d(const float (&v)[M + 2], float (&o)[M])
     if constexpr (M == 4) at_f43(v, o); else at_f63(v, o);
 }
 
-// STORE: 0 = element-wise with bounds checks (any W), 1 = 8-byte stores (W even),
-// 2 = 16-byte stores (F(4,3), W a multiple of 4).  With W a multiple of the store width
-// a tile row is either completely inside the image or completely outside.
+// STORE: 0 = element-wise with bounds checks (any W), 2 = 16-byte stores straight from the
+// registers (F(4,3), W a multiple of 4: neighbouring lanes then write neighbouring 16 bytes
+// and a warp fills whole sectors), 1 = every other even W: the m-float row segments of a
+// tile are 8-byte aligned but 24 (or 16) bytes apart, so that direct 8-byte stores would
+// write every 32-byte sector of y in two or three pieces, and the L2 takes a piece as long
+// as a whole sector (measured: 2.3 sector writes per sector of y, and the kernel bound by
+// them).  The CTA therefore collects its tiles' outputs in shared memory, one array per
+// output row u with the tiles side by side exactly as they lie in the image row, and
+// copies them out with consecutive lanes on consecutive 8 bytes.
 template <int M, int STORE>
 __global__ void __launch_bounds__(128)
 output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geometry g,
                         ScaleTables tab)
 {
     constexpr int NN = M + 2;
+    constexpr int TT = 128;                       // tiles per CTA
+    __shared__ __align__(16) float out_s[STORE == 1 ? M * TT * M : 1];   // [u][tile][v]
+    __shared__ int tile_base[STORE == 1 ? TT : 1];                       // offset of the tile's y[.][.][h0][w0]
+    __shared__ int tile_lim[STORE == 1 ? TT : 1];                        // valid rows * 16 + valid columns
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
     ptx::grid_dependency_wait();   // Y comes from the kernel launched before this one
-    if (t >= g.T) return;
+    const bool live = t < g.T;
+    if (STORE != 1 && !live) return;
 
-    const size_t plane = (size_t)g.K * g.Tp;
-    const float *src = Y + (size_t)k * g.Tp + t;
-    float v[NN][NN];
+    float tmp[M][NN];
+    int h0 = 0, w0 = 0;
+    size_t base = 0;
+    if (live) {
+        const size_t plane = (size_t)g.K * g.Tp;
+        const float *src = Y + (size_t)k * g.Tp + t;
+        float v[NN][NN];
 #pragma unroll
-    for (int i = 0; i < NN; ++i)
+        for (int i = 0; i < NN; ++i)
+#pragma unroll
+            for (int j = 0; j < NN; ++j) {
+                v[i][j] = __ldg(src);
+                src += plane;
+            }
+#pragma unroll
+        for (int i = 0; i < NN; ++i)
+#pragma unroll
+            for (int j = 0; j < NN; ++j) v[i][j] *= tab.out_scale[i * NN + j];
+
+        // columns: tmp[u][j] = sum_i VA[u][i] v[i][j]
 #pragma unroll
         for (int j = 0; j < NN; ++j) {
-            v[i][j] = __ldg(src);
-            src += plane;
+            float col[NN], o[M];
+#pragma unroll
+            for (int i = 0; i < NN; ++i) col[i] = v[i][j];
+            at_1d<M>(col, o);
+#pragma unroll
+            for (int u = 0; u < M; ++u) tmp[u][j] = o[u];
         }
-#pragma unroll
-    for (int i = 0; i < NN; ++i)
-#pragma unroll
-        for (int j = 0; j < NN; ++j) v[i][j] *= tab.out_scale[i * NN + j];
-
-    // columns: tmp[u][j] = sum_i VA[u][i] v[i][j]
-    float tmp[M][NN];
-#pragma unroll
-    for (int j = 0; j < NN; ++j) {
-        float col[NN], o[M];
-#pragma unroll
-        for (int i = 0; i < NN; ++i) col[i] = v[i][j];
-        at_1d<M>(col, o);
-#pragma unroll
-        for (int u = 0; u < M; ++u) tmp[u][j] = o[u];
+        const int tw = t % g.TW;
+        const int tq = t / g.TW;
+        const int th = tq % g.TH;
+        const int img = tq / g.TH;
+        h0 = th * M;
+        w0 = tw * M;
+        base = (((size_t)img * g.K + k) * g.H + h0) * g.W + w0;
     }
 
-    const int tw = t % g.TW;
-    const int tq = t / g.TW;
-    const int th = tq % g.TH;
-    const int img = tq / g.TH;
-    const int h0 = th * M, w0 = tw * M;
-    float *row = y + (((size_t)img * g.K + k) * g.H + h0) * g.W + w0;
-    const bool full_w = (w0 + M <= g.W);
+    if constexpr (STORE == 1) {
+        const int j = threadIdx.x;
+        if (live) {
 #pragma unroll
-    for (int u = 0; u < M; ++u) {
-        float o[M];
-        at_1d<M>(tmp[u], o);
-        if (h0 + u < g.H) {
-            if (STORE == 2 && full_w) {
-                *reinterpret_cast<float4 *>(row) = make_float4(o[0], o[1], o[2], o[3]);
-            } else if (STORE >= 1 && full_w) {
+            for (int u = 0; u < M; ++u) {
+                float o[M];
+                at_1d<M>(tmp[u], o);
+                float2 *dst = reinterpret_cast<float2 *>(out_s + (u * TT + j) * M);
 #pragma unroll
-                for (int v2 = 0; v2 < M; v2 += 2)
-                    *reinterpret_cast<float2 *>(row + v2) = make_float2(o[v2], o[v2 + 1]);
-            } else {
-#pragma unroll
-                for (int v2 = 0; v2 < M; ++v2)
-                    if (w0 + v2 < g.W) row[v2] = o[v2];
+                for (int v2 = 0; v2 < M; v2 += 2) dst[v2 / 2] = make_float2(o[v2], o[v2 + 1]);
             }
         }
-        row += g.W;
+        tile_base[j] = (int)base;
+        tile_lim[j] = live ? (min(M, g.H - h0) * 16 + min(M, g.W - w0)) : 0;
+        __syncthreads();
+        // pair q of row u: tile q / (M/2), columns 2 * (q % (M/2)) and the next
+        constexpr int PPT = M / 2;                // pairs per tile row
+#pragma unroll
+        for (int u = 0; u < M; ++u) {
+            const float2 *row = reinterpret_cast<const float2 *>(out_s + u * TT * M);
+#pragma unroll
+            for (int i = 0; i < PPT; ++i) {
+                const int q = threadIdx.x + i * TT;
+                const int tj = q / PPT, v2 = 2 * (q - tj * PPT);
+                const int lim = tile_lim[tj];
+                if (u < (lim >> 4) && v2 < (lim & 15))      // W even: both columns or none
+                    *reinterpret_cast<float2 *>(y + (size_t)tile_base[tj] + (size_t)u * g.W + v2) = row[q];
+            }
+        }
+    } else {
+        float *row = y + base;
+        const bool full_w = (w0 + M <= g.W);
+#pragma unroll
+        for (int u = 0; u < M; ++u) {
+            float o[M];
+            at_1d<M>(tmp[u], o);
+            if (h0 + u < g.H) {
+                if (STORE == 2 && full_w) {
+                    *reinterpret_cast<float4 *>(row) = make_float4(o[0], o[1], o[2], o[3]);
+                } else {
+#pragma unroll
+                    for (int v2 = 0; v2 < M; ++v2)
+                        if (w0 + v2 < g.W) row[v2] = o[v2];
+                }
+            }
+            row += g.W;
+        }
     }
 }
 
@@ -126,6 +170,15 @@ cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStre
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     const float *Y = plan.ws.Y;
+    // the staged variants want six or more CTAs of 10-19 KB of shared memory per SM
+    static bool carveout_set = false;
+    if (!carveout_set) {
+        cudaFuncSetAttribute(output_transform_kernel<4, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             (int)cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(output_transform_kernel<6, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             (int)cudaSharedmemCarveoutMaxShared);
+        carveout_set = true;
+    }
     // y_dev is 16-byte aligned; rows of an even W keep 8-byte alignment for every tile
     if (g.m == 4) {
         if (g.W % 4 == 0)
