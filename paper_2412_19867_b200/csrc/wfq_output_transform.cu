@@ -1,7 +1,7 @@
 // Output transform y = V_A S_A Y S_A V_A^T (Section 4.1): one thread per
 // (output channel, tile).  Lanes run along the tile index, so the P plane reads of
-// Y[P][K][Tp] are 128-byte coalesced and the m-float row segments written by
-// neighbouring lanes are contiguous in y[N][K][H][W].  Memory-bound: P*4 bytes read
+// Y[P][K][Tp] are 128-byte coalesced; the m-float row segments of neighbouring tiles are
+// contiguous in y[N][K][H][W] and are written in whole sectors.  P*4 bytes read
 // and m*m*4 bytes written per thread against ~150 flops.
 #include "wfq_internal.h"
 #include "wfq_ptx.cuh"
