@@ -41,15 +41,16 @@ __device__ __forceinline__ void at_1d(const float (&v)[M + 2], float (&o)[M])
     if constexpr (M == 4) at_f43(v, o); else at_f63(v, o);
 }
 
-// STORE: 0 = element-wise with bounds checks (any W), 2 = 16-byte stores straight from the
+// STORE: 2 = 16-byte stores straight from the
 // registers (F(4,3), W a multiple of 4: neighbouring lanes then write neighbouring 16 bytes
-// and a warp fills whole sectors), 1 = every other even W: the m-float row segments of a
-// tile are 8-byte aligned but 24 (or 16) bytes apart, so that direct 8-byte stores would
-// write every 32-byte sector of y in two or three pieces, and the L2 takes a piece as long
-// as a whole sector (measured: 2.3 sector writes per sector of y, and the kernel bound by
-// them).  The CTA therefore collects its tiles' outputs in shared memory, one array per
-// output row u with the tiles side by side exactly as they lie in the image row, and
-// copies them out with consecutive lanes on consecutive 8 bytes.
+// and a warp fills whole sectors), 1 = every other even W, 0 = odd W: the m-float row
+// segments of a tile are 24 (or 16) bytes apart, so that direct stores would write every
+// 32-byte sector of y in several pieces, and the L2 takes a piece as long as a whole sector
+// (measured for F(6,3) with 8-byte stores: 2.3 sector writes per sector of y, and the
+// kernel bound by them).  The CTA therefore collects its tiles' outputs in shared memory,
+// one array per output row u with the tiles side by side exactly as they lie in the image
+// row, and copies them out with consecutive lanes on consecutive 8 bytes (even W) or
+// consecutive floats (odd W).
 template <int M, int STORE>
 __global__ void __launch_bounds__(128)
 output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geometry g,
@@ -57,14 +58,14 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
 {
     constexpr int NN = M + 2;
     constexpr int TT = 128;                       // tiles per CTA
-    __shared__ __align__(16) float out_s[STORE == 1 ? M * TT * M : 1];   // [u][tile][v]
-    __shared__ int tile_base[STORE == 1 ? TT : 1];                       // offset of the tile's y[.][.][h0][w0]
-    __shared__ int tile_lim[STORE == 1 ? TT : 1];                        // valid rows * 16 + valid columns
+    __shared__ __align__(16) float out_s[STORE != 2 ? M * TT * M : 1];   // [u][tile][v]
+    __shared__ int tile_base[STORE != 2 ? TT : 1];                       // offset of the tile's y[.][.][h0][w0]
+    __shared__ int tile_lim[STORE != 2 ? TT : 1];                        // valid rows * 16 + valid columns
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int k = blockIdx.y;
     ptx::grid_dependency_wait();   // Y comes from the kernel launched before this one
     const bool live = t < g.T;
-    if (STORE != 1 && !live) return;
+    if (STORE == 2 && !live) return;
 
     float tmp[M][NN];
     int h0 = 0, w0 = 0;
@@ -104,7 +105,7 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
         base = (((size_t)img * g.K + k) * g.H + h0) * g.W + w0;
     }
 
-    if constexpr (STORE == 1) {
+    if constexpr (STORE != 2) {
         const int j = threadIdx.x;
         if (live) {
 #pragma unroll
@@ -119,6 +120,22 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
         tile_base[j] = (int)base;
         tile_lim[j] = live ? (min(M, g.H - h0) * 16 + min(M, g.W - w0)) : 0;
         __syncthreads();
+        if constexpr (STORE == 0) {
+            // float f of row u: tile f / M, column f % M
+#pragma unroll
+            for (int u = 0; u < M; ++u) {
+                const float *row = out_s + u * TT * M;
+#pragma unroll
+                for (int i = 0; i < M; ++i) {
+                    const int f = threadIdx.x + i * TT;
+                    const int tj = f / M, v1 = f - tj * M;
+                    const int lim = tile_lim[tj];
+                    if (u < (lim >> 4) && v1 < (lim & 15))
+                        y[(size_t)tile_base[tj] + (size_t)u * g.W + v1] = row[f];
+                }
+            }
+            return;
+        }
         // pair q of row u: tile q / (M/2), columns 2 * (q % (M/2)) and the next
         constexpr int PPT = M / 2;                // pairs per tile row
 #pragma unroll
@@ -141,7 +158,7 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
             float o[M];
             at_1d<M>(tmp[u], o);
             if (h0 + u < g.H) {
-                if (STORE == 2 && full_w) {
+                if (full_w) {
                     *reinterpret_cast<float4 *>(row) = make_float4(o[0], o[1], o[2], o[3]);
                 } else {
 #pragma unroll
@@ -176,6 +193,10 @@ cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStre
         cudaFuncSetAttribute(output_transform_kernel<4, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
                              (int)cudaSharedmemCarveoutMaxShared);
         cudaFuncSetAttribute(output_transform_kernel<6, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             (int)cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(output_transform_kernel<4, 0>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             (int)cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(output_transform_kernel<6, 0>, cudaFuncAttributePreferredSharedMemoryCarveout,
                              (int)cudaSharedmemCarveoutMaxShared);
         carveout_set = true;
     }
