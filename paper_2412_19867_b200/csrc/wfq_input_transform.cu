@@ -20,8 +20,10 @@
 //            the abs-max serially, derives scale and reciprocal once, rounds with the
 //            1.5*2^23 trick (same result as mul + round-half-even convert; scalar multiply
 //            and add, each rounded) and stores 32 codes per 32-byte store.
-// The abs-max over a group therefore needs no shuffles; for groups of more than 64
-// channels phase 2 reads shared memory twice instead of holding the group in registers.
+// The abs-max over a group of up to 64 channels therefore needs no shuffles; groups of 128
+// or 256 channels are shared by two or four neighbouring lanes (64 channels each, one or two
+// shuffles for the abs-max); other group sizes read shared memory twice instead of holding
+// the group in registers.
 #include <cuda_fp16.h>
 
 #include "wfq_internal.h"
@@ -310,9 +312,10 @@ __device__ __forceinline__ void group_scale(float amax, float &scale, float &inv
 }
 
 // ---- the kernel ----------------------------------------------------------------------
-// GSR > 0: compile-time group size held in registers during phase 2 (32 or 64);
-// GSR == 0: any group size, phase 2 reads shared memory twice.
-template <int M, typename Tin, int GSR>
+// GSR > 0: channels a thread holds in registers during phase 2 (32 or 64); a group is GSR *
+// SPLIT channels, SPLIT neighbouring lanes share it and exchange their abs-max by shuffle.
+// GSR == 0: any group size, one thread per group, phase 2 reads shared memory twice.
+template <int M, typename Tin, int GSR, int SPLIT>
 __global__ void __launch_bounds__(K1_THREADS, 4)
 input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
                        float *__restrict__ sX, Geometry g, ScaleTables tab, K1Params prm)
@@ -327,7 +330,7 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int NWARP = K1_THREADS / 32;
     const int cb32 = prm.CB >> 5;
-    const int gs = GSR > 0 ? GSR : g.gs;
+    const int gs = GSR > 0 ? GSR * SPLIT : g.gs;
     const int ng = prm.CB / gs;
 
     // item -> (tile row, chunk of tiles, channel block); channel blocks vary fastest so
@@ -378,32 +381,54 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
         // X = Z * (caller's per-position factor) is formed here, one rounding, as the
         // quantizer's input; then abs-max, scale, reciprocal and codes.
         const int g_base = c_base / gs;
-        const int tasks = ntile * ng * P;
-        for (int task = threadIdx.x; task < tasks; task += K1_THREADS) {
-            const int q = task / P, p = task - q * P;
-            const int tl = q / ng, grp = q - tl * ng;
-            const int t = srow * g.TW + tw0 + tl;
-            const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs);
-            int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
-            const float sp = tab.in_scale[p];
-            const float2 sp2 = make_float2(sp, sp);
-            float scale, inv;
-            if constexpr (GSR > 0) {
+        if constexpr (GSR > 0) {
+            // whole warps walk the loop so that the lanes sharing a group can shuffle
+            const int tasks = ntile * ng * P * SPLIT;
+            for (int base = 0; base < tasks; base += K1_THREADS) {
+                const int task = base + (int)threadIdx.x;
+                const bool act = task < tasks;          // the lanes of a group are all in or all out
+                const int tk = act ? task : 0;
+                const int part = tk % SPLIT, rest = tk / SPLIT;
+                const int q = rest / P, p = rest - q * P;
+                const int tl = q / ng, grp = q - tl * ng;
+                const int t = srow * g.TW + tw0 + tl;
+                const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs +
+                                                                     part * GSR);
+                int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs + part * GSR;
+                const float sp = tab.in_scale[p];
+                const float2 sp2 = make_float2(sp, sp);
                 float4 v[GSR / 4];
                 float amax = 0.f;
-    #pragma unroll
+#pragma unroll
                 for (int k = 0; k < GSR / 4; ++k) {
                     v[k] = scale4(src[k], sp2);
                     amax = absmax4(amax, v[k]);
                 }
+                if constexpr (SPLIT >= 2) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                if constexpr (SPLIT >= 4) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+                float scale, inv;
                 group_scale(amax, scale, inv);
-    #pragma unroll
-                for (int k = 0; k < GSR / 32; ++k)        // 32 codes = one full sector per store
-                    st_global_v8_b32(dst + 32 * k, codes4(v[8 * k], inv), codes4(v[8 * k + 1], inv),
-                                     codes4(v[8 * k + 2], inv), codes4(v[8 * k + 3], inv),
-                                     codes4(v[8 * k + 4], inv), codes4(v[8 * k + 5], inv),
-                                     codes4(v[8 * k + 6], inv), codes4(v[8 * k + 7], inv));
-            } else {
+                if (act) {
+#pragma unroll
+                    for (int k = 0; k < GSR / 32; ++k)        // 32 codes = one full sector per store
+                        st_global_v8_b32(dst + 32 * k, codes4(v[8 * k], inv), codes4(v[8 * k + 1], inv),
+                                         codes4(v[8 * k + 2], inv), codes4(v[8 * k + 3], inv),
+                                         codes4(v[8 * k + 4], inv), codes4(v[8 * k + 5], inv),
+                                         codes4(v[8 * k + 6], inv), codes4(v[8 * k + 7], inv));
+                    if (part == 0) sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
+                }
+            }
+        } else {
+            const int tasks = ntile * ng * P;
+            for (int task = threadIdx.x; task < tasks; task += K1_THREADS) {
+                const int q = task / P, p = task - q * P;
+                const int tl = q / ng, grp = q - tl * ng;
+                const int t = srow * g.TW + tw0 + tl;
+                const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs);
+                int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
+                const float sp = tab.in_scale[p];
+                const float2 sp2 = make_float2(sp, sp);
+                float scale, inv;
                 float amax = 0.f;
                 for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2));
                 group_scale(amax, scale, inv);
@@ -413,14 +438,14 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
                                      codes4(scale4(src[8 * k + 3], sp2), inv), codes4(scale4(src[8 * k + 4], sp2), inv),
                                      codes4(scale4(src[8 * k + 5], sp2), inv), codes4(scale4(src[8 * k + 6], sp2), inv),
                                      codes4(scale4(src[8 * k + 7], sp2), inv));
+                sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
             }
-            sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
         }
         __syncthreads();   // Z and this strip buffer are free again
     }
 }
 
-template <int M, typename Tin, int GSR>
+template <int M, typename Tin, int GSR, int SPLIT>
 cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stream)
 {
     const Geometry &g = plan.geo;
@@ -455,7 +480,7 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
     const size_t smem = smem_bytes();
     prm.NCH = (g.TW + prm.TB - 1) / prm.TB;
 
-    auto kern = input_transform_kernel<M, Tin, GSR>;
+    auto kern = input_transform_kernel<M, Tin, GSR, SPLIT>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -478,9 +503,11 @@ template <int M, typename Tin>
 cudaError_t dispatch_gs(const wfq_plan &plan, const void *x, cudaStream_t s)
 {
     const int gs = plan.geo.gs;
-    if (gs == 32) return launch_k1<M, Tin, 32>(plan, x, s);
-    if (gs == 64) return launch_k1<M, Tin, 64>(plan, x, s);
-    return launch_k1<M, Tin, 0>(plan, x, s);
+    if (gs == 32) return launch_k1<M, Tin, 32, 1>(plan, x, s);
+    if (gs == 64) return launch_k1<M, Tin, 64, 1>(plan, x, s);
+    if (gs == 128) return launch_k1<M, Tin, 64, 2>(plan, x, s);
+    if (gs == 256) return launch_k1<M, Tin, 64, 4>(plan, x, s);
+    return launch_k1<M, Tin, 0, 1>(plan, x, s);
 }
 
 }  // namespace
