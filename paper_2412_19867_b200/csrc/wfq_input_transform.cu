@@ -471,6 +471,9 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
     // strip buffer is used only where it does not cost a resident CTA (registers allow four).
     prm.dbuf = 0;
     while (prm.TB > 1 && smem_bytes() > 113 * 1024) --prm.TB;
+    // the same number of chunks per tile row with evenly sized chunks (four tiles: 2 + 2, not 3 + 1)
+    prm.NCH = (g.TW + prm.TB - 1) / prm.TB;
+    prm.TB = (g.TW + prm.NCH - 1) / prm.NCH;
     {
         const size_t per_sm = 227 * 1024, one = smem_bytes() + 1024;
         const size_t two = one + prm.strip_bytes;
@@ -478,7 +481,6 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
         if (n2 >= 1 && n2 == n1) prm.dbuf = 1;
     }
     const size_t smem = smem_bytes();
-    prm.NCH = (g.TW + prm.TB - 1) / prm.TB;
 
     auto kern = input_transform_kernel<M, Tin, GSR, SPLIT>;
     if (smem > 48 * 1024) {
