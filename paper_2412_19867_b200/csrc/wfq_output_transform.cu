@@ -52,7 +52,7 @@ __device__ __forceinline__ void at_1d(const float (&v)[M + 2], float (&o)[M])
 // row, and copies them out with consecutive lanes on consecutive 8 bytes (even W) or
 // consecutive floats (odd W).
 template <int M, int STORE>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, M == 6 ? 7 : 8)
 output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geometry g,
                         ScaleTables tab)
 {
