@@ -75,6 +75,21 @@ typedef enum {
     WFQ_BUF_STATUS = 5  /* int32 status[4]: {code, where, block, aux} (plan-owned) */
 } wfq_buffer_t;
 
+/* Test and profiling switches of wfq_plan_set_debug_option. */
+typedef enum {
+    WFQ_DEBUG_WAIT_CYCLES = 0,      /* limit of every device-side wait in SM clock cycles
+                                       (default 2e9, about a second; at least 1000) */
+    WFQ_DEBUG_SKIP_INPUT_ITEM = 1,  /* work item whose input strip the tensor-core input
+                                       transform's producer does not load (-1 = none): the
+                                       waits for it run out, the kernel records
+                                       WFQ_ERR_TIMEOUT in the status word and ends by itself */
+    WFQ_DEBUG_GENERIC_INPUT_TRANSFORM = 2, /* nonzero: always use the cp.async input-transform
+                                       kernel, also where the tensor-core one applies */
+    WFQ_DEBUG_SKIP_GEMM_STAGE = 3   /* operand stage (counted from 0) whose loads the first
+                                       CTA of the contraction kernel does not issue (-1 =
+                                       none); same purpose as WFQ_DEBUG_SKIP_INPUT_ITEM */
+} wfq_debug_option_t;
+
 /*
  * Create a plan for one layer: x[N][C][H][W] -> y[N][K][H][W] evaluated as F(m,3)
  * (Section 3.1: output tile m x m, filter r x r, input tile (m+r-1)^2).
@@ -115,9 +130,14 @@ wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t byte
  *   sG_host  host, n floats, diagonal of S_G (NULL = standard scales)
  *   sA_host  host, n floats, diagonal of S_A (NULL = 1/(sB*sG), Eq. scaling_condition,
  *            evaluated in fp64 and rounded to fp32)
- * All scales must be finite and nonzero (signs are allowed).  Allocates the
- * plan-owned Wq/sW buffers on first use (cudaMalloc), runs on `stream`, and may be
- * called again to replace the filters.
+ * All scales must be finite and nonzero (signs are allowed).  The first call on a plan
+ * allocates the plan-owned Wq/sW buffers and the status word with cudaMalloc (which may
+ * synchronise the device); every call takes the fp32 temporary between its two kernels
+ * from the stream-ordered allocator (cudaMallocAsync / cudaFreeAsync on `stream`), so
+ * later calls neither block nor synchronise.  Asynchronous on `stream`; may be called
+ * again to replace the filters.  The first library call that meets a device (this one or
+ * wfq_plan_set_workspace) also sets that device's kernel attributes; make it outside any
+ * stream capture.
  */
 wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const float *sB_host,
                                  const float *sG_host, const float *sA_host, void *stream);
@@ -153,6 +173,8 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
  * when a call starts (harmless, every element that is read is written first by the
  * same call, so nothing needs clearing), and two calls whose kernels can overlap on
  * the GPU (different streams, or different host threads) race on it.  Serialise them.
+ * The looked-up address is cached per device ordinal for the life of the process;
+ * cudaDeviceReset invalidates it, so do not call this function after a device reset.
  */
 #define WFQ_STATIC_SCRATCH_FLOATS (4u * 1024u * 1024u)
 wfq_status_t wfq_quantize_filters_static(const float *w_dev, int K, int C, int m, int group_size,
@@ -164,8 +186,10 @@ wfq_status_t wfq_quantize_filters_static(const float *w_dev, int K, int C, int m
  * contraction with per-group dequantization, output transform.
  *   x_dev  device, [N][C][H][W] in the plan's input dtype, 4-byte aligned
  *   y_dev  device, fp32 [N][K][H][W], 16-byte aligned
- * Three kernels are enqueued on `stream`; no host synchronisation.  Requires a
- * workspace and prepared filters (WFQ_ERR_NOT_PREPARED otherwise).
+ * Three kernels are enqueued on `stream`; no host synchronisation and no other runtime
+ * call, except that a TMA descriptor of x is re-encoded (host only) when x_dev differs
+ * from the previous call's.  Requires a workspace and prepared filters
+ * (WFQ_ERR_NOT_PREPARED otherwise).
  */
 wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev, void *stream);
 
@@ -198,6 +222,23 @@ wfq_status_t wfq_output_transform(wfq_plan_t *plan, float *y_dev, void *stream);
  * P*T*K*G elements.
  */
 wfq_status_t wfq_debug_gemm_acc32(wfq_plan_t *plan, int32_t *acc_dev, void *stream);
+
+/*
+ * Measurement aid: the rate of the int8 tensor pipe as this library drives it.  Enqueues on
+ * `stream` one CTA per SM, each issuing `mmas_per_sm` (a multiple of 4) accumulating
+ * tcgen05.mma kind::i8 instructions of shape 128 x n_cols x 32 (n_cols in {64, 128, 256}) on
+ * operands resident in shared memory, and stores in *ops (host) the number of integer
+ * operations (2 per multiply-add) the launch performs; the caller times the launch.  No
+ * global memory is read or written.  Needs prepared filters (for the status word).
+ */
+wfq_status_t wfq_debug_int8_mma_rate(wfq_plan_t *plan, int n_cols, int mmas_per_sm, long long *ops,
+                                     void *stream);
+
+/*
+ * Set a test/profiling switch of the plan (see wfq_debug_option_t).  Host only.
+ * WFQ_ERR_INVALID_ARG for an unknown option or a value outside its range.
+ */
+wfq_status_t wfq_plan_set_debug_option(wfq_plan_t *plan, wfq_debug_option_t option, long long value);
 
 /*
  * Device address and size of an internal buffer (see wfq_buffer_t for layouts).

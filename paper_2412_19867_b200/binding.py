@@ -16,6 +16,8 @@ WFQ_ERR_NOT_PREPARED, WFQ_ERR_CUDA, WFQ_ERR_TIMEOUT, WFQ_ERR_SCRATCH_TOO_SMALL =
 WFQ_STATIC_SCRATCH_FLOATS = 4 * 1024 * 1024
 WFQ_F32, WFQ_F16 = 0, 1
 WFQ_BUF_XQ, WFQ_BUF_SX, WFQ_BUF_WQ, WFQ_BUF_SW, WFQ_BUF_Y, WFQ_BUF_STATUS = range(6)
+WFQ_DEBUG_WAIT_CYCLES, WFQ_DEBUG_SKIP_INPUT_ITEM, WFQ_DEBUG_GENERIC_INPUT_TRANSFORM = range(3)
+WFQ_DEBUG_SKIP_GEMM_STAGE = 3
 
 # every symbol include/wfq.h declares
 EXPORTS = [
@@ -24,7 +26,7 @@ EXPORTS = [
     "wfq_conv_forward_host", "wfq_input_transform_quantize", "wfq_gemm_dequantize",
     "wfq_output_transform", "wfq_debug_gemm_acc32", "wfq_debug_get",
     "wfq_check_device_status", "wfq_plan_destroy", "wfq_status_string", "wfq_version",
-    "wfq_quantize_filters_static",
+    "wfq_quantize_filters_static", "wfq_plan_set_debug_option", "wfq_debug_int8_mma_rate",
 ]
 
 _lib = None
@@ -62,6 +64,8 @@ def load():
     lib.wfq_check_device_status.argtypes = [vp, vp, ctypes.POINTER(ci)]
     lib.wfq_plan_destroy.argtypes = [vp]
     lib.wfq_quantize_filters_static.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
+    lib.wfq_plan_set_debug_option.argtypes = [vp, ci, ctypes.c_longlong]
+    lib.wfq_debug_int8_mma_rate.argtypes = [vp, ci, ci, ctypes.POINTER(ctypes.c_longlong), vp]
     lib.wfq_status_string.argtypes = [ci]
     lib.wfq_status_string.restype = ctypes.c_char_p
     lib.wfq_version.restype = ci
@@ -158,6 +162,18 @@ def wfq_quantize_filters_static(w_dev, K, C, m, group_size, sG, wq_dev, sw_dev, 
     keep, pg = _host_floats(sG)
     _check(load().wfq_quantize_filters_static(w_dev, K, C, m, group_size, pg, wq_dev, sw_dev, stream),
            "wfq_quantize_filters_static")
+
+
+def wfq_plan_set_debug_option(plan, option, value):
+    _check(load().wfq_plan_set_debug_option(plan, option, value), "wfq_plan_set_debug_option")
+
+
+def wfq_debug_int8_mma_rate(plan, n_cols, mmas_per_sm, stream=0):
+    """Enqueues the tensor-pipe rate kernel; returns the integer operations it performs."""
+    ops = ctypes.c_longlong(0)
+    _check(load().wfq_debug_int8_mma_rate(plan, n_cols, mmas_per_sm, ctypes.byref(ops), stream),
+           "wfq_debug_int8_mma_rate")
+    return ops.value
 
 
 def wfq_plan_destroy(plan):

@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "wfq_internal.h"
@@ -37,12 +38,46 @@ wfq_status_t ready_to_run(const wfq_plan *plan)
 
 size_t in_elem_bytes(const wfq_plan *plan) { return plan->in_dtype == WFQ_F16 ? 2 : 4; }
 
+// Kernel attributes (dynamic shared-memory limits, carveouts) are per device and are set
+// the first time a plan meets the device; launches then make no other runtime call.
+constexpr int kMaxDevices = 64;
+std::mutex g_setup_mutex;
+bool g_device_ready[kMaxDevices];
+
+wfq_status_t bind_device(wfq_plan *plan)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return WFQ_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return WFQ_ERR_UNSUPPORTED;
+    if (plan->device == dev && plan->sm_count > 0) return WFQ_OK;
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return WFQ_ERR_CUDA;
+    if (major != 10) return WFQ_ERR_UNSUPPORTED;
+    {
+        std::lock_guard<std::mutex> lock(g_setup_mutex);
+        if (!g_device_ready[dev]) {
+            if (wfq::setup_input_transform() != cudaSuccess || wfq::setup_input_transform_tc() != cudaSuccess ||
+                wfq::setup_gemm() != cudaSuccess || wfq::setup_output_transform() != cudaSuccess)
+                return WFQ_ERR_CUDA;
+            g_device_ready[dev] = true;
+        }
+    }
+    plan->device = dev;
+    plan->sm_count = sms;
+    wfq::plan_input_transform(*plan);
+    wfq::plan_input_transform_tc(*plan);
+    return WFQ_OK;
+}
+
 }  // namespace
 
 namespace wfq {
 
-bool encode_tmap_bytes3d(CUtensorMap *map, const void *base, int inner, int rows, int planes,
-                         int box_rows)
+bool encode_tmap(CUtensorMap *map, CUtensorMapDataType dtype, int rank, const void *base,
+                 const unsigned long long *dims, const unsigned long long *strides,
+                 const unsigned *box, CUtensorMapSwizzle swizzle)
 {
     typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
@@ -57,15 +92,27 @@ bool encode_tmap_bytes3d(CUtensorMap *map, const void *base, int inner, int rows
             return false;
         encode = reinterpret_cast<EncodeFn>(fn);
     }
-    cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)planes};
-    cuuint64_t strides[2] = {(cuuint64_t)inner, (cuuint64_t)inner * (cuuint64_t)rows};
-    cuuint32_t box[3] = {128u, (cuuint32_t)box_rows, 1u};
-    cuuint32_t estr[3] = {1u, 1u, 1u};
-    CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), dims,
-                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    if (rank < 1 || rank > 3) return false;
+    cuuint64_t d[3], st[2];
+    cuuint32_t bx[3], estr[3] = {1u, 1u, 1u};
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
+    CUresult r = encode(map, dtype, (cuuint32_t)rank, const_cast<void *>(base), d, st, bx, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
+}
+
+bool encode_tmap_bytes3d(CUtensorMap *map, const void *base, int inner, int rows, int planes,
+                         int box_rows)
+{
+    const unsigned long long dims[3] = {(unsigned long long)inner, (unsigned long long)rows,
+                                        (unsigned long long)planes};
+    const unsigned long long strides[2] = {(unsigned long long)inner,
+                                           (unsigned long long)inner * (unsigned long long)rows};
+    const unsigned box[3] = {128u, (unsigned)box_rows, 1u};
+    return encode_tmap(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, base, dims, strides, box,
+                       CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 }  // namespace wfq
@@ -134,6 +181,12 @@ wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype)
     if (!plan) return WFQ_ERR_INVALID_ARG;
     if (dtype != WFQ_F32 && dtype != WFQ_F16) return WFQ_ERR_INVALID_ARG;
     plan->in_dtype = dtype;
+    plan->host_chunks = 0;            // chunk starts are aligned for the element size
+    plan->tmap_x_base = nullptr;
+    if (plan->sm_count > 0) {
+        wfq::plan_input_transform(*plan);
+        wfq::plan_input_transform_tc(*plan);
+    }
     return WFQ_OK;
 }
 
@@ -144,6 +197,8 @@ wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t byte
     if (!plan || !dev_ptr) return WFQ_ERR_INVALID_ARG;
     if (bytes < plan->ws.total || (reinterpret_cast<uintptr_t>(dev_ptr) & 1023u) != 0)
         return WFQ_ERR_INVALID_ARG;
+    wfq_status_t bs = bind_device(plan);
+    if (bs != WFQ_OK) return bs;
     wfq::Workspace &ws = plan->ws;
     char *base = static_cast<char *>(dev_ptr);
     ws.Xq = reinterpret_cast<int8_t *>(base);
@@ -185,13 +240,9 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
             plan->tables.out_scale[i * g.n + j] = (float)(plan->sA[i] * plan->sA[j]);
         }
 
-    cudaError_t e = cudaGetDevice(&plan->device);
-    if (e != cudaSuccess) return WFQ_ERR_CUDA;
-    cudaDeviceProp prop;
-    e = cudaGetDeviceProperties(&prop, plan->device);
-    if (e != cudaSuccess) return WFQ_ERR_CUDA;
-    if (prop.major != 10) return WFQ_ERR_UNSUPPORTED;
-    plan->sm_count = prop.multiProcessorCount;
+    wfq_status_t bs = bind_device(plan);
+    if (bs != WFQ_OK) return bs;
+    cudaError_t e;
 
     const size_t wq_bytes = (size_t)g.P * g.K * g.C;
     const size_t sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
@@ -207,11 +258,14 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
         if ((e = cudaMemsetAsync(plan->status, 0, 4 * sizeof(int), as_stream(stream))) != cudaSuccess)
             return WFQ_ERR_CUDA;
     }
-    float *w32 = nullptr;  // fp32 transformed filters, released after quantization
-    if ((e = cudaMalloc(&w32, wq_bytes * sizeof(float))) != cudaSuccess) return cuda_status(e);
-    e = wfq::launch_filter_prep(*plan, w_dev, w32, as_stream(stream));
-    cudaError_t e2 = cudaStreamSynchronize(as_stream(stream));
-    cudaFree(w32);
+    // fp32 transformed filters between the two kernels: stream-ordered allocation, released
+    // in stream order after the quantization kernel, so the call neither blocks nor holds
+    // the temporary (four times the size of Wq) any longer than the kernels need it
+    void *w32 = nullptr;
+    if ((e = cudaMallocAsync(&w32, wq_bytes * sizeof(float), as_stream(stream))) != cudaSuccess)
+        return cuda_status(e);
+    e = wfq::launch_filter_prep(*plan, w_dev, static_cast<float *>(w32), as_stream(stream));
+    cudaError_t e2 = cudaFreeAsync(w32, as_stream(stream));
     if (e != cudaSuccess || e2 != cudaSuccess) return WFQ_ERR_CUDA;
 
     plan->tmap_wq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_wq, plan->Wq, g.C, g.K, g.P,
@@ -242,6 +296,18 @@ wfq_status_t wfq_debug_gemm_acc32(wfq_plan_t *plan, int32_t *acc_dev, void *stre
     if (s != WFQ_OK) return s;
     if (!acc_dev) return WFQ_ERR_INVALID_ARG;
     return cuda_status(wfq::launch_gemm(*plan, acc_dev, as_stream(stream), false));
+}
+
+wfq_status_t wfq_debug_int8_mma_rate(wfq_plan_t *plan, int n_cols, int mmas_per_sm, long long *ops,
+                                     void *stream)
+{
+    if (!plan || !ops) return WFQ_ERR_INVALID_ARG;
+    if (!plan->prepared) return WFQ_ERR_NOT_PREPARED;       // needs the status word and the device
+    if ((n_cols != 64 && n_cols != 128 && n_cols != 256) || mmas_per_sm < 4 || mmas_per_sm > (1 << 24) ||
+        mmas_per_sm % 4 != 0)
+        return WFQ_ERR_INVALID_ARG;
+    *ops = (long long)plan->sm_count * mmas_per_sm * 2LL * 128 * n_cols * 32;
+    return cuda_status(wfq::launch_mma_peak(*plan, n_cols, mmas_per_sm, as_stream(stream)));
 }
 
 wfq_status_t wfq_output_transform(wfq_plan_t *plan, float *y_dev, void *stream)
@@ -292,7 +358,8 @@ static wfq_status_t setup_host_pipeline(wfq_plan *plan)
             plan->sub[s]->borrowed = true;
         }
         wfq_plan *q = plan->sub[s];
-        q->in_dtype = plan->in_dtype;
+        wfq_plan_set_input_dtype(q, plan->in_dtype);
+        q->debug_force_generic_k1 = plan->debug_force_generic_k1;
         // same orientation of the contraction as the whole batch: identical arithmetic
         q->gemm_swap = plan->gemm_swap;
         q->gemm_bn = plan->gemm_bn;
@@ -303,7 +370,7 @@ static wfq_status_t setup_host_pipeline(wfq_plan *plan)
         q->Wq = plan->Wq; q->sW = plan->sW; q->status = plan->status;
         q->tables = plan->tables;
         q->tmap_wq = plan->tmap_wq; q->tmap_wq_ok = plan->tmap_wq_ok;
-        q->device = plan->device; q->sm_count = plan->sm_count;
+        q->wait_cycles = plan->wait_cycles;
         q->prepared = true;
         if (!plan->host_stream[s] &&
             cudaStreamCreateWithFlags(&plan->host_stream[s], cudaStreamNonBlocking) != cudaSuccess)
@@ -342,26 +409,34 @@ wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *
         for (int i = 0; i < 2; ++i)
             if (cudaStreamWaitEvent(plan->host_stream[i], plan->host_event[2], 0) != cudaSuccess)
                 return WFQ_ERR_CUDA;
-        for (int c = 0; c < chunks; ++c) {
+        wfq_status_t err = WFQ_OK;
+        for (int c = 0; c < chunks && err == WFQ_OK; ++c) {
             cudaStream_t cs = plan->host_stream[c & 1];
             char *xd = static_cast<char *>(plan->x_stage) + (size_t)c * xc;
             float *yd = plan->y_stage + (size_t)c * (yc / sizeof(float));
             if (cudaMemcpyAsync(xd, static_cast<const char *>(x_host) + (size_t)c * xc, xc,
-                                cudaMemcpyHostToDevice, cs) != cudaSuccess)
-                return WFQ_ERR_CUDA;
-            s = wfq_conv_forward(plan->sub[c & 1], xd, yd, cs);
-            if (s != WFQ_OK) return s;
-            if (cudaMemcpyAsync(reinterpret_cast<char *>(y_host) + (size_t)c * yc, yd, yc,
+                                cudaMemcpyHostToDevice, cs) != cudaSuccess) {
+                err = WFQ_ERR_CUDA;
+                break;
+            }
+            err = wfq_conv_forward(plan->sub[c & 1], xd, yd, cs);
+            if (err == WFQ_OK &&
+                cudaMemcpyAsync(reinterpret_cast<char *>(y_host) + (size_t)c * yc, yd, yc,
                                 cudaMemcpyDeviceToHost, cs) != cudaSuccess)
-                return WFQ_ERR_CUDA;
+                err = WFQ_ERR_CUDA;
         }
-        // and the caller's stream continues after both of them
+        // The caller's stream continues after both internal streams; on an error the
+        // copies already queued are waited for as well, so that nothing writes y_host
+        // after this (synchronous) call has returned.
         for (int i = 0; i < 2; ++i) {
             if (cudaEventRecord(plan->host_event[i], plan->host_stream[i]) != cudaSuccess ||
-                cudaStreamWaitEvent(st, plan->host_event[i], 0) != cudaSuccess)
-                return WFQ_ERR_CUDA;
+                cudaStreamWaitEvent(st, plan->host_event[i], 0) != cudaSuccess) {
+                cudaStreamSynchronize(plan->host_stream[i]);
+                if (err == WFQ_OK) err = WFQ_ERR_CUDA;
+            }
         }
-        return cuda_status(cudaStreamSynchronize(st));
+        const cudaError_t se = cudaStreamSynchronize(st);
+        return err != WFQ_OK ? err : cuda_status(se);
     }
 
     if ((e = cudaMemcpyAsync(plan->x_stage, x_host, xb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
@@ -371,6 +446,36 @@ wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *
     if ((e = cudaMemcpyAsync(y_host, plan->y_stage, yb, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
         return WFQ_ERR_CUDA;
     return cuda_status(cudaStreamSynchronize(st));
+}
+
+wfq_status_t wfq_plan_set_debug_option(wfq_plan_t *plan, wfq_debug_option_t option, long long value)
+{
+    if (!plan) return WFQ_ERR_INVALID_ARG;
+    switch (option) {
+        case WFQ_DEBUG_WAIT_CYCLES:
+            if (value < 1000) return WFQ_ERR_INVALID_ARG;
+            plan->wait_cycles = value;
+            break;
+        case WFQ_DEBUG_SKIP_INPUT_ITEM:
+            if (value < -1 || value > 0x7fffffff) return WFQ_ERR_INVALID_ARG;
+            plan->debug_skip_item = (int)value;
+            break;
+        case WFQ_DEBUG_GENERIC_INPUT_TRANSFORM:
+            plan->debug_force_generic_k1 = value != 0;
+            break;
+        case WFQ_DEBUG_SKIP_GEMM_STAGE:
+            if (value < -1 || value > 0x7fffffff) return WFQ_ERR_INVALID_ARG;
+            plan->debug_skip_gemm_stage = (int)value;
+            break;
+        default:
+            return WFQ_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < 2; ++i)
+        if (plan->sub[i]) {
+            plan->sub[i]->wait_cycles = plan->wait_cycles;
+            plan->sub[i]->debug_force_generic_k1 = plan->debug_force_generic_k1;
+        }
+    return WFQ_OK;
 }
 
 wfq_status_t wfq_debug_get(wfq_plan_t *plan, wfq_buffer_t which, void **dev_ptr, size_t *bytes)

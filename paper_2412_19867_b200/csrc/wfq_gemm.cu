@@ -49,7 +49,6 @@ constexpr int A_BYTES = BM * BK;
 constexpr int NUM_EPI_WARPS = 4;
 constexpr int FIRST_EPI_WARP = 4;
 constexpr int NUM_THREADS = 32 * (FIRST_EPI_WARP + NUM_EPI_WARPS);
-constexpr long long WAIT_CYCLES = 2000000000LL;   // ~1 s at 2 GHz
 
 struct Shared {
     uint64_t full[NSTAGES];        // operands of a stage have landed
@@ -73,48 +72,6 @@ struct Cfg {
                                          (size_t)NSLOT * SLOT_SCALE_FLOATS * sizeof(float) + sizeof(Shared);
 };
 
-// Bounded mbarrier wait.  Returns false (and records `where`) on timeout or when
-// another role of this CTA already gave up.  The common case, a phase that has already
-// completed, is one try_wait inline; the waiting loop is kept out of line so that the
-// role loops stay short (their instructions sit on the critical path between MMAs).
-// In the loop the bare try_wait suspends the thread in hardware for up to a
-// millisecond; clock and abort flag are looked at every 64 tries.
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, Shared *sh, int *status, int where)
-{
-    long long t0 = 0;
-#pragma unroll 1
-    for (uint32_t it = 1;; ++it) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0) {
-            if (sh->abort) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            if (now - t0 > WAIT_CYCLES) {
-                sh->abort = 1;
-                if (atomicCAS(status, 0, (int)WFQ_ERR_TIMEOUT) == 0) {
-                    status[1] = where;
-                    status[2] = (int)blockIdx.x;
-                    status[3] = (int)parity;
-                }
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Shared *sh, int *status,
-                                             int where)
-{
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    return wait_slow(bar, parity, sh, status, where);
-}
-
-// Bounded wait for copies that may still be in flight when a role gives up.
-__device__ __forceinline__ void drain(uint32_t bar, uint32_t parity)
-{
-    const long long t0 = clock64();
-    while (!ptx::mbar_try_wait(bar, parity) && clock64() - t0 < WAIT_CYCLES / 16) { }
-}
-
 struct GemmArgs {
     const float *row_scale;   // [P][G][row_pitch]: sX (normal) or sW (swapped)
     const float *col_scale;   // [P][G][col_pitch]: sW (normal) or sX (swapped)
@@ -124,6 +81,8 @@ struct GemmArgs {
     float *Y;                 // [P][K][Tp]
     int32_t *acc_dump;        // [P][T][K][G] or null
     int *status;
+    long long wait_cycles;    // limit of every mbarrier wait (about a second by default)
+    int debug_skip_stage;     // >= 0: CTA 0's producer skips the loads of this stage (test hook)
 };
 
 // MMA issue loop for the common shapes in which the chunks tile a stage exactly
@@ -135,7 +94,7 @@ struct GemmArgs {
 template <int BN, int GSTEPS, int CGT>
 __device__ __forceinline__ void mma_issue_aligned(Shared *sh, uint32_t tiles_lo, uint32_t tmem_base,
                                                   int units, int KB, int last_slices, int lane,
-                                                  int *status)
+                                                  const WaitCtx &ctx)
 {
     using C = Cfg<BN>;
     constexpr int CHUNK_STEPS = GSTEPS * CGT;            // MMAs per chunk
@@ -150,14 +109,14 @@ __device__ __forceinline__ void mma_issue_aligned(Shared *sh, uint32_t tiles_lo,
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
         for (int kb = 0; kb < KB; ++kb) {
             const int nslice = kb == KB - 1 ? last_slices : BK / UK;
-            if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8u * stage, phase, sh, status, kWaitSmemFull)))
+            if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8u * stage, phase, ctx, kWaitSmemFull)))
                 return;
             const uint32_t a_lo = tiles_lo + (uint32_t)(stage * (C::STAGE_BYTES >> 4));
             const uint32_t b_lo = a_lo + (uint32_t)(A_BYTES >> 4);
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
                 if (c * CHUNK_STEPS < nslice) {           // the chunk has at least one group
-                    if (!__all_sync(0xffffffffu, wait_bounded(free0 + 8u * slot, sphase ^ 1u, sh, status,
+                    if (!__all_sync(0xffffffffu, wait_bounded(free0 + 8u * slot, sphase ^ 1u, ctx,
                                                               kWaitTmemEmpty)))
                         return;
                     ptx::tc_fence_after();
@@ -215,7 +174,7 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int gs_steps = g.gs / UK;              // MMAs per group
     const int cg = a.cg;                         // groups per chunk
     const int nchunk = (g.G + cg - 1) / cg;      // chunks per unit
-    int *status = a.status;
+    const WaitCtx ctx{&sh->abort, a.status, a.wait_cycles};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NSTAGES; ++s) {
@@ -258,10 +217,10 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
             const int nt = u % NT, mt = (u / NT) % MT, p = u / (NT * MT);
             for (int kb = 0; kb < KB; ++kb) {
-                ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, sh,
-                                                          status, kWaitSmemEmpty));
+                ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, ctx,
+                                                          kWaitSmemEmpty));
                 if (!ok) break;
-                if (lane == 0) {
+                if (lane == 0 && !(blockIdx.x == 0 && issued == a.debug_skip_stage)) {
                     const uint32_t bar = ptx::smem_u32(&sh->full[stage]);
                     const uint32_t a_dst = ptx::smem_u32(tiles + (size_t)stage * C::STAGE_BYTES);
                     ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
@@ -280,7 +239,7 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const long long n = issued < NSTAGES ? issued : NSTAGES;
             for (long long i = 0; i < n; ++i) {
                 if (--s < 0) { s = NSTAGES - 1; ph ^= 1u; }
-                drain(ptx::smem_u32(&sh->full[s]), ph);
+                drain(ptx::smem_u32(&sh->full[s]), ph, a.wait_cycles / 16);
             }
         }
     } else if (warp == 1) {
@@ -298,14 +257,14 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         bool ok = true;
         // shapes whose chunks tile a stage exactly take the straight-line issue loop
         if (gs_steps == 2 && cg == 2) {
-            mma_issue_aligned<BN, 2, 2>(sh, tiles_lo, tmem_base, units, KB, last_slices, lane, status);
+            mma_issue_aligned<BN, 2, 2>(sh, tiles_lo, tmem_base, units, KB, last_slices, lane, ctx);
             ok = false;
         } else if (gs_steps == 4 && cg == 1) {
-            mma_issue_aligned<BN, 4, 1>(sh, tiles_lo, tmem_base, units, KB, last_slices, lane, status);
+            mma_issue_aligned<BN, 4, 1>(sh, tiles_lo, tmem_base, units, KB, last_slices, lane, ctx);
             ok = false;
         } else if (gs_steps == 1 && cg == C::CG_MAX && C::CG_MAX <= 4) {
             mma_issue_aligned<BN, 1, (C::CG_MAX <= 4 ? C::CG_MAX : 4)>(sh, tiles_lo, tmem_base, units, KB,
-                                                                    last_slices, lane, status);
+                                                                    last_slices, lane, ctx);
             ok = false;
         }
         for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
@@ -313,7 +272,7 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             int in_group = 0;      // MMA step within the group
             uint32_t dcol = 0;     // TMEM column of the current group
             for (int kb = 0; kb < KB && ok; ++kb) {
-                ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->full[stage]), phase, sh, status,
+                ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->full[stage]), phase, ctx,
                                                           kWaitSmemFull));
                 if (!ok) break;
                 ptx::tc_fence_after();
@@ -325,7 +284,7 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (step == 0) {
                         // start of a chunk: its TMEM slot must have been drained
                         ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->slot_free[slot]),
-                                                                  sphase ^ 1u, sh, status, kWaitTmemEmpty));
+                                                                  sphase ^ 1u, ctx, kWaitTmemEmpty));
                         if (!ok) break;
                         ptx::tc_fence_after();
                         dcol = tmem_base + (uint32_t)(slot * SLOT_COLS);
@@ -366,7 +325,7 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 for (int ch = 0; ch < nchunk; ++ch) {
                     const int g0 = ch * cg, ng = min(cg, g.G - g0);
                     ok = __all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->slot_free[slot]), sphase ^ 1u,
-                                                              sh, status, kWaitScaleEmpty));
+                                                              ctx, kWaitScaleEmpty));
                     if (!ok) break;
                     const uint32_t bar = ptx::smem_u32(&sh->scale_full[slot]);
                     const uint32_t dst = ptx::smem_u32(scales + (size_t)slot * C::SLOT_SCALE_FLOATS);
@@ -393,7 +352,7 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const long long n = issued < NSLOT ? issued : NSLOT;
                 for (long long i = 0; i < n; ++i) {
                     if (--s < 0) { s = NSLOT - 1; ph ^= 1u; }
-                    drain(ptx::smem_u32(&sh->scale_full[s]), ph);
+                    drain(ptx::smem_u32(&sh->scale_full[s]), ph, a.wait_cycles / 16);
                 }
             }
         }
@@ -418,11 +377,11 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
             for (int ch = 0; ch < nchunk && ok; ++ch) {
                 const int g0 = ch * cg, ng = min(cg, g.G - g0);
-                if (!wait_bounded(ptx::smem_u32(&sh->acc_full[slot]), sphase, sh, status, kWaitTmemFull)) {
+                if (!wait_bounded(ptx::smem_u32(&sh->acc_full[slot]), sphase, ctx, kWaitTmemFull)) {
                     ok = false; break;
                 }
                 if constexpr (!DUMP) {
-                    if (!wait_bounded(ptx::smem_u32(&sh->scale_full[slot]), sphase, sh, status,
+                    if (!wait_bounded(ptx::smem_u32(&sh->scale_full[slot]), sphase, ctx,
                                       kWaitScaleFull)) { ok = false; break; }
                 }
                 if (active) {
@@ -528,14 +487,13 @@ cudaError_t launch_variant(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t
     a.Y = plan.ws.Y;
     a.acc_dump = acc_dump;
     a.status = plan.status;
+    a.wait_cycles = plan.wait_cycles;
+    a.debug_skip_stage = plan.debug_skip_gemm_stage;
     const int MT = (a.rows + BM - 1) / BM, NT = (a.cols + BN - 1) / BN;
     const int units = g.P * MT * NT;
     const int slots = 2 * plan.sm_count;          // two CTAs per SM
     const int grid = units < slots ? units : slots;
     auto kern = gemm_dequant_kernel<BN, SWAP, DUMP>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(NUM_THREADS);
@@ -551,7 +509,103 @@ cudaError_t launch_variant(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t
     return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, a, g);
 }
 
+// ---- tensor-pipe rate of tcgen05.mma kind::i8 -----------------------------------------
+// One CTA per SM issues `mmas` accumulating 128 x BN x 32 MMAs on operands that stay in
+// shared memory (no global traffic), then waits (bounded) for the last one.  Timed by the
+// caller with events: grid * mmas * 2 * 128 * BN * 32 operations.
+struct PeakShared { uint64_t done; uint32_t tmem_base; volatile int abort; };
+
+template <int BN>
+__global__ void __launch_bounds__(128, 1) mma_peak_kernel(int mmas, int *status, long long wait_cycles)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *tiles = reinterpret_cast<unsigned char *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int BYTES = (BM + BN) * BK;
+    PeakShared *sh = reinterpret_cast<PeakShared *>(tiles + BYTES);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = threadIdx.x; i < BYTES / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(tiles)[i] = 0x01010101u;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_u32(&sh->done), 1);
+        sh->abort = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 0) {
+        ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), BN < 32 ? 32 : BN);
+        ptx::tmem_relinquish();
+    }
+    ptx::fence_proxy_async_smem();
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+    if (warp == 0) {
+        const WaitCtx ctx{&sh->abort, status, wait_cycles};
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
+            constexpr uint32_t dhi = ptx::smem_desc_sw128_hi();
+            const uint32_t a_lo = ptx::smem_desc_sw128_lo(ptx::smem_u32(tiles));
+            const uint32_t b_lo = a_lo + (uint32_t)(A_BYTES >> 4);
+            for (int i = 0; i < mmas; i += 4) {
+                ptx::umma_i8_lo<true>(tmem, a_lo, b_lo, dhi, idesc);
+                ptx::umma_i8_lo<true>(tmem, a_lo + 2, b_lo + 2, dhi, idesc);
+                ptx::umma_i8_lo<true>(tmem, a_lo + 4, b_lo + 4, dhi, idesc);
+                ptx::umma_i8_lo<true>(tmem, a_lo + 6, b_lo + 6, dhi, idesc);
+            }
+            ptx::umma_commit(ptx::smem_u32(&sh->done));
+        }
+        __syncwarp();
+        wait_bounded(ptx::smem_u32(&sh->done), 0, ctx, kWaitTmemFull);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, BN < 32 ? 32 : BN);
+    }
+}
+
+template <int BN>
+cudaError_t launch_peak(int grid, int mmas, int *status, long long wait_cycles, cudaStream_t stream)
+{
+    const int smem = 1024 + (BM + BN) * BK + (int)sizeof(PeakShared);
+    cudaError_t e = cudaFuncSetAttribute(mma_peak_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    mma_peak_kernel<BN><<<grid, 128, smem, stream>>>(mmas, status, wait_cycles);
+    return cudaGetLastError();
+}
+
+template <int BN, bool SWAP, bool DUMP>
+cudaError_t setup_variant()
+{
+    return cudaFuncSetAttribute(gemm_dequant_kernel<BN, SWAP, DUMP>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<BN>::SMEM_BYTES);
+}
+
 }  // namespace
+
+// One-time attribute setting for the kernels of this file (per device).
+cudaError_t setup_gemm()
+{
+    cudaError_t e = setup_variant<32, true, true>();
+    if (e == cudaSuccess) e = setup_variant<32, true, false>();
+    if (e == cudaSuccess) e = setup_variant<64, true, true>();
+    if (e == cudaSuccess) e = setup_variant<64, true, false>();
+    if (e == cudaSuccess) e = setup_variant<64, false, true>();
+    if (e == cudaSuccess) e = setup_variant<64, false, false>();
+    return e;
+}
+
+cudaError_t launch_mma_peak(const wfq_plan &plan, int n_cols, int mmas, cudaStream_t stream)
+{
+    const int grid = plan.sm_count;
+    switch (n_cols) {
+        case 64: return launch_peak<64>(grid, mmas, plan.status, plan.wait_cycles, stream);
+        case 128: return launch_peak<128>(grid, mmas, plan.status, plan.wait_cycles, stream);
+        case 256: return launch_peak<256>(grid, mmas, plan.status, plan.wait_cycles, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
 
 int gemm_block_m() { return BM; }
 

@@ -34,18 +34,6 @@ namespace {
 constexpr int K1_THREADS = 128;
 constexpr int K1_WP = 16;        // staged columns per row (image columns w_base .. w_base+15)
 
-struct K1Params {
-    int TB;            // tiles per work item
-    int NCH;           // chunks of TB tiles per tile row
-    int NCB;           // channel blocks (C / CB)
-    int items;         // work items: N * TH * NCH * NCB
-    int CB;            // channels per work item (a multiple of the group size)
-    int CS;            // shared-memory channel stride of the strip (elements)
-    int strip_bytes;   // bytes of the strip, rounded up to 16
-    int pair;          // 1: rows can be copied as aligned element pairs
-    int dbuf;          // 1: two strip buffers, the next item is staged during this one
-};
-
 // ---- 1-D input transforms with the standard B^T ------------------------------------
 
 // F(4,3): rows [4,0,-5,0,1,0] [0,-4,-4,1,1,0] [0,4,-4,-1,1,0] [0,-2,-1,2,1,0]
@@ -445,14 +433,71 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
     }
 }
 
+// Resident CTAs per SM and the attribute calls need the kernel symbol: one entry per
+// instantiation.
+template <int M, typename Tin, int GSR, int SPLIT>
+int k1_resident(size_t smem)
+{
+    return resident_ctas_per_sm(input_transform_kernel<M, Tin, GSR, SPLIT>, K1_THREADS, smem, 32);
+}
+
+template <int M, typename Tin, int GSR, int SPLIT>
+cudaError_t k1_setup()
+{
+    auto kern = input_transform_kernel<M, Tin, GSR, SPLIT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                (int)cudaSharedmemCarveoutMaxShared);
+}
+
 template <int M, typename Tin, int GSR, int SPLIT>
 cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stream)
 {
+    const K1Params &prm = plan.k1;
+    input_transform_kernel<M, Tin, GSR, SPLIT><<<prm.grid, K1_THREADS, prm.smem, stream>>>(
+        static_cast<const Tin *>(x_dev), plan.ws.Xq, plan.ws.sX, plan.geo, plan.tables, prm);
+    return cudaGetLastError();
+}
+
+// What to do with the instantiation that serves (m, dtype, group size).
+enum K1Op { kK1Launch, kK1Resident, kK1Setup };
+
+template <int M, typename Tin>
+long long k1_by_gs(K1Op op, int gs, const wfq_plan *plan, const void *x, cudaStream_t s, size_t smem)
+{
+#define WFQ_K1_CASE(GSR, SPLIT)                                                        \
+    switch (op) {                                                                      \
+        case kK1Launch: return (long long)launch_k1<M, Tin, GSR, SPLIT>(*plan, x, s);  \
+        case kK1Resident: return k1_resident<M, Tin, GSR, SPLIT>(smem);                \
+        default: return (long long)k1_setup<M, Tin, GSR, SPLIT>();                     \
+    }
+    if (gs == 32) { WFQ_K1_CASE(32, 1) }
+    if (gs == 64) { WFQ_K1_CASE(64, 1) }
+    if (gs == 128) { WFQ_K1_CASE(64, 2) }
+    if (gs == 256) { WFQ_K1_CASE(64, 4) }
+    WFQ_K1_CASE(0, 1)
+#undef WFQ_K1_CASE
+}
+
+long long k1_op(K1Op op, int m, bool f16, int gs, const wfq_plan *plan, const void *x, cudaStream_t s,
+                size_t smem)
+{
+    if (m == 4)
+        return f16 ? k1_by_gs<4, __half>(op, gs, plan, x, s, smem) : k1_by_gs<4, float>(op, gs, plan, x, s, smem);
+    return f16 ? k1_by_gs<6, __half>(op, gs, plan, x, s, smem) : k1_by_gs<6, float>(op, gs, plan, x, s, smem);
+}
+
+}  // namespace
+
+// Work-item shape, shared-memory layout and grid of the cp.async kernel for this plan.
+void plan_input_transform(wfq_plan &plan)
+{
     const Geometry &g = plan.geo;
-    constexpr int NN = M + 2;
-    constexpr int P = NN * NN;
-    const int esz = (int)sizeof(Tin);
-    K1Params prm;
+    const bool f16 = plan.in_dtype == WFQ_F16;
+    const int NN = g.n, P = g.P, M = g.m;
+    const int esz = f16 ? 2 : 4;
+    K1Params &prm = plan.k1;
     prm.TB = (K1_WP - 3) / M;                      // 2 tiles for F(6,3), 3 for F(4,3)
     prm.CB = g.gs;
     if (g.gs == 32 && g.C % 64 == 0) prm.CB = 64;  // two groups per CTA
@@ -463,7 +508,7 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
     else if (cs % 2 == 0) cs += 1;
     prm.CS = cs;
     prm.strip_bytes = (prm.CB * cs * esz + 15) / 16 * 16;
-    prm.pair = (g.W % 2 == 0) && (reinterpret_cast<uintptr_t>(x_dev) % 4 == 0);
+    prm.pair = (g.W % 2 == 0);                     // x is 4-byte aligned (checked by the entry points)
     auto smem_bytes = [&]() {
         return (1 + prm.dbuf) * (size_t)prm.strip_bytes + (size_t)prm.TB * P * (prm.CB + 4) * sizeof(float);
     };
@@ -480,48 +525,53 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
         const size_t n1 = per_sm / one < 4 ? per_sm / one : 4, n2 = per_sm / two < 4 ? per_sm / two : 4;
         if (n2 >= 1 && n2 == n1) prm.dbuf = 1;
     }
-    const size_t smem = smem_bytes();
-
-    auto kern = input_transform_kernel<M, Tin, GSR, SPLIT>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
+    prm.smem = (int)smem_bytes();
     prm.NCB = g.C / prm.CB;
     prm.items = g.N * g.TH * prm.NCH * prm.NCB;
     // persistent CTAs: as many as fit on the device at once
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                         (int)cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-    const int per_sm = resident_ctas_per_sm(kern, K1_THREADS, smem, 32);
-    const int resident = per_sm * plan.sm_count;
-    const int grid = prm.items < resident ? prm.items : resident;
-    kern<<<grid, K1_THREADS, smem, stream>>>(static_cast<const Tin *>(x_dev), plan.ws.Xq, plan.ws.sX, g,
-                                             plan.tables, prm);
-    return cudaGetLastError();
+    const int per_sm = (int)k1_op(kK1Resident, M, f16, g.gs, nullptr, nullptr, nullptr, (size_t)prm.smem);
+    const int resident = per_sm * (plan.sm_count > 0 ? plan.sm_count : 1);
+    prm.grid = prm.items < resident ? prm.items : resident;
 }
 
-template <int M, typename Tin>
-cudaError_t dispatch_gs(const wfq_plan &plan, const void *x, cudaStream_t s)
+cudaError_t setup_input_transform()
 {
-    const int gs = plan.geo.gs;
-    if (gs == 32) return launch_k1<M, Tin, 32, 1>(plan, x, s);
-    if (gs == 64) return launch_k1<M, Tin, 64, 1>(plan, x, s);
-    if (gs == 128) return launch_k1<M, Tin, 64, 2>(plan, x, s);
-    if (gs == 256) return launch_k1<M, Tin, 64, 4>(plan, x, s);
-    return launch_k1<M, Tin, 0, 1>(plan, x, s);
+    const int sizes[5] = {32, 64, 128, 256, 96};
+    for (int m = 4; m <= 6; m += 2)
+        for (int f16 = 0; f16 < 2; ++f16)
+            for (int gs : sizes) {
+                cudaError_t e = (cudaError_t)k1_op(kK1Setup, m, f16 != 0, gs, nullptr, nullptr, nullptr, 0);
+                if (e != cudaSuccess) return e;
+            }
+    return cudaSuccess;
 }
 
-}  // namespace
-
-cudaError_t launch_input_transform(const wfq_plan &plan, const void *x_dev, cudaStream_t stream)
+cudaError_t launch_input_transform(wfq_plan &plan, const void *x_dev, cudaStream_t stream)
 {
-    const bool f16 = plan.in_dtype == WFQ_F16;
-    if (plan.geo.m == 4)
-        return f16 ? dispatch_gs<4, __half>(plan, x_dev, stream)
-                   : dispatch_gs<4, float>(plan, x_dev, stream);
-    return f16 ? dispatch_gs<6, __half>(plan, x_dev, stream)
-               : dispatch_gs<6, float>(plan, x_dev, stream);
+    const Geometry &g = plan.geo;
+    // tensor-core kernel: fp16 input that a TMA tensor map (16-byte aligned base) can describe
+    if (plan.k1tc.use && !plan.debug_force_generic_k1 && (reinterpret_cast<uintptr_t>(x_dev) & 15u) == 0) {
+        if (plan.k1tc.mode != 2 && plan.tmap_x_base != x_dev) {
+            const unsigned long long hw = (unsigned long long)g.H * g.W;
+            bool ok;
+            if (plan.k1tc.mode == 0) {
+                const unsigned long long dims[3] = {(unsigned long long)g.W, (unsigned long long)g.H,
+                                                    (unsigned long long)g.N * g.C};
+                const unsigned long long strides[2] = {(unsigned long long)g.W * 2, hw * 2};
+                ok = encode_tmap(&plan.tmap_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, x_dev, dims, strides,
+                                 plan.k1tc.box, CU_TENSOR_MAP_SWIZZLE_NONE);
+            } else {
+                const unsigned long long dims[2] = {hw, (unsigned long long)g.N * g.C};
+                const unsigned long long strides[1] = {hw * 2};
+                ok = encode_tmap(&plan.tmap_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, x_dev, dims, strides,
+                                 plan.k1tc.box, CU_TENSOR_MAP_SWIZZLE_NONE);
+            }
+            if (!ok) return cudaErrorInvalidValue;
+            plan.tmap_x_base = x_dev;
+        }
+        return launch_input_transform_tc(plan, x_dev, stream);
+    }
+    return (cudaError_t)k1_op(kK1Launch, g.m, plan.in_dtype == WFQ_F16, g.gs, &plan, x_dev, stream, 0);
 }
 
 }  // namespace wfq

@@ -21,7 +21,13 @@ enum WaitId : int {
     kWaitTmemFull = 4,    // epilogue waiting for a finished accumulator
     kWaitDrain = 5,       // teardown waiting for copies in flight
     kWaitScaleEmpty = 6,  // scale loader waiting for a free ring slot
-    kWaitScaleFull = 7    // epilogue waiting for a group's scales
+    kWaitScaleFull = 7,   // epilogue waiting for a group's scales
+    kWaitStripEmpty = 8,  // input transform: TMA producer waiting for a free strip buffer
+    kWaitStripFull = 9,   // input transform: im2col warps waiting for a strip
+    kWaitPairEmpty = 10,  // input transform: im2col warps waiting for a free operand tile
+    kWaitPairFull = 11,   // input transform: MMA issuer waiting for operand tiles
+    kWaitAccEmpty = 12,   // input transform: MMA issuer waiting for a drained accumulator
+    kWaitAccFull = 13     // input transform: quantizer waiting for an accumulator
 };
 
 // Geometry and scale tables handed to the kernels by value.
@@ -38,6 +44,34 @@ struct ScaleTables {
     float in_scale[kMaxP];   // (sB_i/sBstd_i)*(sB_j/sBstd_j): applied after the
                              // standard-scaled integer/rational input transform
     float out_scale[kMaxP];  // sA_i*sA_j: applied before the output transform
+};
+
+// Launch parameters of the cp.async input-transform kernel (any dtype, any shape),
+// computed once per plan.
+struct K1Params {
+    int TB;            // tiles per work item
+    int NCH;           // chunks of TB tiles per tile row
+    int NCB;           // channel blocks (C / CB)
+    int items;         // work items: N * TH * NCH * NCB
+    int CB;            // channels per work item (a multiple of the group size)
+    int CS;            // shared-memory channel stride of the strip (elements)
+    int strip_bytes;   // bytes of the strip, rounded up to 16
+    int pair;          // 1: rows can be copied as aligned element pairs
+    int dbuf;          // 1: two strip buffers, the next item is staged during this one
+    int smem, grid;    // dynamic shared memory and CTAs of the launch
+};
+
+// Launch parameters of the tensor-core input-transform kernel (fp16 inputs, groups of 32
+// or 64 channels, C a multiple of 64, shapes a TMA or bulk copy can stage).
+struct K1TcPlan {
+    bool use = false;
+    int mode = 0;            // 0: 3-D tiled TMA (W, H, N*C); 1: 2-D tiled TMA (H*W, N*C); 2: bulk copy
+    int TBW = 0, NCHUNK = 0, NCB = 0, items = 0;
+    int CS = 0, RS = 0;      // strip strides in elements: channel, patch row
+    int strip_bytes = 0, nstrip = 0, nbp = 0;
+    int nbox = 1, rpb = 0, box_elems = 0;   // mode 1: boxes per strip, rows per box, elements per box row
+    int smem = 0, grid = 0;
+    unsigned box[3] = {0, 0, 0};
 };
 
 struct Workspace {
@@ -68,6 +102,16 @@ struct wfq_plan {
     double sB[wfq::kMaxN], sG[wfq::kMaxN], sA[wfq::kMaxN];
     wfq::ScaleTables tables;
 
+    // launch parameters derived from the geometry, the dtype and the device (plan_launches)
+    wfq::K1Params k1;
+    wfq::K1TcPlan k1tc;
+    CUtensorMap tmap_x;        // the input tensor as the tensor-core input transform stages it
+    const void *tmap_x_base = nullptr;   // x pointer tmap_x was encoded for
+    long long wait_cycles = 2000000000LL;   // limit of every device-side wait (~1 s)
+    int debug_skip_item = -1;  // >= 0: the input transform's producer skips this work item
+    int debug_skip_gemm_stage = -1;   // >= 0: the contraction's producer (CTA 0) skips this stage
+    int debug_force_generic_k1 = 0;   // 1: always use the cp.async input-transform kernel
+
     CUtensorMap tmap_xq;       // Xq as (C, T, P) bytes, 128B-swizzled boxes
     CUtensorMap tmap_wq;       // Wq as (C, K, P)
     bool tmap_xq_ok = false, tmap_wq_ok = false;
@@ -92,9 +136,26 @@ namespace wfq {
 // launch; none synchronises.
 cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *scratch_w32,
                                cudaStream_t stream);
-cudaError_t launch_input_transform(const wfq_plan &plan, const void *x_dev, cudaStream_t stream);
+cudaError_t launch_input_transform(wfq_plan &plan, const void *x_dev, cudaStream_t stream);
+cudaError_t launch_input_transform_tc(const wfq_plan &plan, const void *x_dev, cudaStream_t stream);
+
+// Per-plan launch parameters (host only, no device work) and per-device one-time kernel
+// attributes (shared-memory sizes and carveouts).
+void plan_input_transform(wfq_plan &plan);
+void plan_input_transform_tc(wfq_plan &plan);
+cudaError_t setup_input_transform();
+cudaError_t setup_input_transform_tc();
+cudaError_t setup_gemm();
+cudaError_t setup_output_transform();
+
+// General tiled tensor map (rank 2 or 3, no interleave, zero fill outside the tensor).
+// `strides` are in bytes for dimensions 1.. (rank - 1 entries).
+bool encode_tmap(CUtensorMap *map, CUtensorMapDataType dtype, int rank, const void *base,
+                 const unsigned long long *dims, const unsigned long long *strides,
+                 const unsigned *box, CUtensorMapSwizzle swizzle);
 cudaError_t launch_gemm(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t stream, bool pdl);
 cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStream_t stream, bool pdl);
+cudaError_t launch_mma_peak(const wfq_plan &plan, int n_cols, int mmas, cudaStream_t stream);
 
 // Builds a 3-D byte tensor map (inner extent `inner`, rows, planes) with a
 // (128, box_rows, 1) box and 128-byte swizzle.  Returns false on failure.

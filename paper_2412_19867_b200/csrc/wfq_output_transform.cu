@@ -173,6 +173,22 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
 
 }  // namespace
 
+// One-time attribute setting (per device): the staged variants want six or more CTAs of
+// 10-19 KB of shared memory per SM.
+cudaError_t setup_output_transform()
+{
+    const int carve = (int)cudaSharedmemCarveoutMaxShared;
+    cudaError_t e = cudaFuncSetAttribute(output_transform_kernel<4, 1>,
+                                         cudaFuncAttributePreferredSharedMemoryCarveout, carve);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(output_transform_kernel<6, 1>, cudaFuncAttributePreferredSharedMemoryCarveout, carve);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(output_transform_kernel<4, 0>, cudaFuncAttributePreferredSharedMemoryCarveout, carve);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(output_transform_kernel<6, 0>, cudaFuncAttributePreferredSharedMemoryCarveout, carve);
+    return e;
+}
+
 cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStream_t stream, bool pdl)
 {
     const Geometry &g = plan.geo;
@@ -187,19 +203,6 @@ cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStre
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     const float *Y = plan.ws.Y;
-    // the staged variants want six or more CTAs of 10-19 KB of shared memory per SM
-    static bool carveout_set = false;
-    if (!carveout_set) {
-        cudaFuncSetAttribute(output_transform_kernel<4, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             (int)cudaSharedmemCarveoutMaxShared);
-        cudaFuncSetAttribute(output_transform_kernel<6, 1>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             (int)cudaSharedmemCarveoutMaxShared);
-        cudaFuncSetAttribute(output_transform_kernel<4, 0>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             (int)cudaSharedmemCarveoutMaxShared);
-        cudaFuncSetAttribute(output_transform_kernel<6, 0>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             (int)cudaSharedmemCarveoutMaxShared);
-        carveout_set = true;
-    }
     // y_dev is 16-byte aligned; rows of an even W keep 8-byte alignment for every tile
     if (g.m == 4) {
         if (g.W % 4 == 0)

@@ -83,6 +83,24 @@ __device__ __forceinline__ void st_global_v8(float *p, float a, float b, float c
                  : "memory");
 }
 
+// 2-D tiled load.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                            int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+// Makes this thread's earlier shared-memory writes (generic proxy) visible to the
+// asynchronous proxy (TMA, tcgen05.mma operand reads).
+__device__ __forceinline__ void fence_proxy_async_smem()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 // ---- programmatic dependent launch ---------------------------------------------------
 // Blocks until the grid this one was launched behind has completed and its writes are
 // visible (no-op for an ordinary launch).
@@ -156,6 +174,28 @@ __device__ __forceinline__ void umma_i8_lo(uint32_t d_tmem, uint32_t a_lo, uint3
             ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc));
     }
 }
+// D[tmem] (+)= A[smem] * B[smem], fp16 x fp16 -> fp32 (K = 16 per instruction), descriptors
+// given as for umma_i8_lo.
+template <bool ACCUMULATE>
+__device__ __forceinline__ void umma_f16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                            uint32_t desc_hi, uint32_t idesc)
+{
+    if constexpr (ACCUMULATE) {
+        asm volatile(
+            "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "setp.eq.b32 p, 0, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc));
+    } else {
+        asm volatile(
+            "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "setp.ne.b32 p, 0, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc));
+    }
+}
 // Arrive on `bar` once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
@@ -174,6 +214,29 @@ __device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
           "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
           "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+// 64 columns in two x32 loads into one register array (no wait in between).
+__device__ __forceinline__ void tmem_ld_x64(uint32_t taddr, uint32_t (&r)[64])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+        "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+        "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+          "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
+          "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]),
+          "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]),
+          "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]),
+          "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]),
+          "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]),
+          "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]),
+          "=r"(r[62]), "=r"(r[63])
         : "r"(taddr)
         : "memory");
 }
@@ -231,5 +294,62 @@ __host__ __device__ constexpr uint32_t idesc_i8(int M, int N)
            ((uint32_t)(M >> 4) << 24);
 }
 
+// Instruction descriptor for kind::f16 with fp16 A and B (both K-major), fp32 D:
+//   [4,6) D format = 1 (f32), [7,10) A format = 0 (f16), [10,13) B format = 0 (f16),
+//   [17,23) N >> 3, [24,29) M >> 4.
+__host__ __device__ constexpr uint32_t idesc_f16(int M, int N)
+{
+    return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
 }  // namespace ptx
+
+// ---- bounded waits ------------------------------------------------------------------
+// Every mbarrier wait of the tensor-core kernels has a time limit.  On expiry the thread
+// sets the CTA's abort flag, records {WFQ_ERR_TIMEOUT, where, block, parity} in the plan's
+// status word (first writer wins) and returns false; the other roles see the flag and
+// stop as well, the CTA drains its copies, frees TMEM and exits.
+struct WaitCtx {
+    volatile int *abort;    // shared memory, one per CTA
+    int *status;            // global, int32[4]
+    long long limit;        // clock cycles
+};
+
+// The waiting loop is kept out of line so that the role loops stay short.  The bare
+// try_wait suspends the thread in hardware for up to a millisecond; clock and abort flag
+// are looked at every 64 tries.
+static __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const WaitCtx &ctx, int where)
+{
+    long long t0 = 0;
+#pragma unroll 1
+    for (uint32_t it = 1;; ++it) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0 || ctx.limit < 100000000LL) {
+            if (*ctx.abort) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > ctx.limit) {
+                *ctx.abort = 1;
+                if (atomicCAS(ctx.status, 0, 6 /* WFQ_ERR_TIMEOUT */) == 0) {
+                    ctx.status[1] = where;
+                    ctx.status[2] = (int)blockIdx.x;
+                    ctx.status[3] = (int)parity;
+                }
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, const WaitCtx &ctx, int where)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    return wait_slow(bar, parity, ctx, where);
+}
+// Bounded wait for copies that may still be in flight when a role gives up.
+__device__ __forceinline__ void drain(uint32_t bar, uint32_t parity, long long limit)
+{
+    const long long t0 = clock64();
+    while (!ptx::mbar_try_wait(bar, parity) && clock64() - t0 < limit) { }
+}
+
 }  // namespace wfq

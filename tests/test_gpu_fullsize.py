@@ -12,8 +12,9 @@ from paper_2412_19867_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-FULL = ([L for L in wl.config_layers(2)] + [wl.config_layers(3)[i] for i in (0, 5, 8, 9)]
-        + wl.config_layers(4) + [wl.config_layers(5)[i] for i in (0, 1, 3, 5, 8)])
+# every configured layer: 1 + 4 + 12 + 3 + 10 (configuration 1 is also run in full by
+# test_gpu_parity.py)
+FULL = [L for cfg in (2, 3, 4, 5) for L in wl.config_layers(cfg)]
 
 
 @pytest.mark.parametrize("layer", FULL, ids=lambda L: L.name)

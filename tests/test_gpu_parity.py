@@ -49,6 +49,16 @@ SMALL = [
     # four groups per chunk; with whole 128-channel stages and with a 32-channel last stage
     Layer(1, 128, 128, 8, 8, 4, 32, "f16", "silu_outlier", "kaiming_chan", 4, 0, 5),
     Layer(2, 160, 192, 8, 8, 4, 32, "f16", "silu_outlier", "kaiming_chan", 4, 0, 6),
+    # groups that straddle the 128-channel stages of the contraction, several groups per unit,
+    # a partial last stage; both orientations
+    Layer(1, 192, 40, 13, 13, 6, 96, "f16", "silu_outlier", "kaiming_chan", 4, 0, 7),
+    Layer(1, 320, 64, 8, 8, 4, 160, "f16", "silu_outlier", "kaiming_chan", 4, 0, 8),    # swapped
+    Layer(2, 512, 64, 12, 12, 4, 256, "f16", "silu_outlier", "kaiming_chan", 4, 0, 9),
+    # tensor-core input transform: column chunks with a ragged last chunk (3-D boxes), whole
+    # tile rows in several boxes, an odd number of operand tiles per CTA, groups of 32
+    Layer(1, 64, 32, 24, 136, 4, 64, "f16", "silu_outlier", "kaiming_chan", 5, 0, 1),   # W = 136: chunks
+    Layer(1, 128, 32, 20, 64, 6, 32, "f16", "silu_outlier", "kaiming_chan", 5, 5, 1),   # 11 tiles per row
+    Layer(5, 64, 32, 10, 16, 6, 64, "f16", "relu_heavy", "kaiming", 2, 0, 2),           # 3 tiles per row
 ]
 
 
@@ -116,6 +126,76 @@ def test_host_buffer_entry_point_in_chunks_matches_device_one():
         assert torch.equal(yh, y_dev)
     conv.check_status()
     conv.close()
+
+
+def test_input_transform_kernels_agree():
+    """The tensor-core input transform and the cp.async one (selected by a debug option)
+    against the oracle and against each other on the same layer, and a misaligned x
+    (which the tensor-core kernel's TMA descriptor cannot take) falls back by itself."""
+    import torch
+    from oracle import oracle as orc
+    from paper_2412_19867_b200 import binding as b
+    from tests.gpu_util import make_conv, codes_close, scales_close
+    L = Layer(2, 128, 32, 24, 24, 6, 64, "f16", "silu_outlier", "kaiming_chan", 5, 6, 2)
+    conv, (x, w, sB, sG) = make_conv(L)
+    ref = orc.wfq(x, w[:1], L.m, L.gs, sB=sB, sG=sG)
+    xbuf = torch.zeros(x.size + 8, dtype=torch.float16, device="cuda")
+    got = []
+    for force, offset in ((0, 0), (1, 0), (0, 2)):          # offset in elements: 4-byte aligned only
+        xd = xbuf[offset:offset + x.size].view(x.shape)
+        xd.copy_(torch.from_numpy(x))
+        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_GENERIC_INPUT_TRANSFORM, force)
+        conv.buffer(b.WFQ_BUF_XQ).fill_(99)
+        b.wfq_input_transform_quantize(conv.plan, xd.data_ptr(), conv._stream())
+        torch.cuda.synchronize()
+        conv.check_status()
+        xq = conv.buffer(b.WFQ_BUF_XQ).cpu().numpy()
+        codes_close(xq, ref.Xq)
+        scales_close(conv.buffer(b.WFQ_BUF_SX).cpu().numpy()[:, :, :conv.T], ref.sX.transpose(0, 2, 1))
+        got.append(xq)
+    assert np.mean(got[0] != got[1]) <= 1e-4
+    assert np.array_equal(got[1], got[2])                   # both from the cp.async kernel
+    conv.close()
+
+
+def test_bounded_waits_run_out_and_report():
+    """A load that never arrives: the waits for it end by themselves after the (shortened)
+    limit, the kernel records WFQ_ERR_TIMEOUT with the id of the wait in the status word,
+    drains, frees its tensor memory and returns; a fresh plan then computes correctly."""
+    import torch
+    from paper_2412_19867_b200 import binding as b
+    from tests.gpu_util import make_conv, max_rel
+    from oracle import oracle as orc
+    L = Layer(1, 64, 64, 16, 16, 4, 64, "f16", "silu_outlier", "kaiming_chan", 9, 5, 0)
+    # (option, value, stage call, expected wait ids)
+    cases = [(b.WFQ_DEBUG_SKIP_INPUT_ITEM, 1, "k1", {9}),    # im2col warps wait for the strip
+             (b.WFQ_DEBUG_SKIP_GEMM_STAGE, 0, "k2", {2})]    # MMA issuer waits for operands
+    for option, value, stage, want in cases:
+        conv, (x, w, sB, sG) = make_conv(L)
+        xd = torch.from_numpy(x).cuda()
+        y = conv.forward(xd)                                  # a clean call first
+        torch.cuda.synchronize()
+        conv.check_status()
+        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_WAIT_CYCLES, 2_000_000)   # about 1 ms
+        b.wfq_plan_set_debug_option(conv.plan, option, value)
+        if stage == "k1":
+            b.wfq_input_transform_quantize(conv.plan, xd.data_ptr(), conv._stream())
+        else:
+            b.wfq_gemm_dequantize(conv.plan, conv._stream())
+        torch.cuda.synchronize()                              # the kernel ended by itself
+        st, where = b.wfq_check_device_status(conv.plan, conv._stream())
+        assert st == b.WFQ_ERR_TIMEOUT, (stage, st)
+        assert where in want, (stage, where)
+        conv.close()
+        # the context is intact: a fresh plan gives the right answer
+        conv, _ = make_conv(L, (x, w, sB, sG))
+        y2 = conv.forward(xd)
+        torch.cuda.synchronize()
+        conv.check_status()
+        assert torch.equal(y, y2)
+        ref = orc.wfq(x, w, L.m, L.gs, sB=sB, sG=sG)
+        assert max_rel(y2.cpu().numpy(), ref.y) <= 2e-3
+        conv.close()
 
 
 def test_misaligned_or_null_device_pointers_are_rejected():

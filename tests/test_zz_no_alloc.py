@@ -35,6 +35,11 @@ def _both_ways(layer):
     codes_close(got_q.cpu().numpy(), want_q)
     scales_close(got_s.cpu().numpy(), want_s, rtol=1e-6)
     assert np.array_equal(got_q.cpu().numpy(), want_q)         # same kernels: identical
+    # and directly against the CPU oracle's offline filter path
+    from oracle import oracle as orc
+    ref = orc.prepare_filters(w, layer.m, layer.gs, orc.matrices(layer.m, sB, sG))
+    codes_close(got_q.cpu().numpy(), ref.Wq)
+    scales_close(got_s.cpu().numpy(), ref.sW.transpose(0, 2, 1), rtol=1e-6)
     conv.close()
 
 
