@@ -1,17 +1,23 @@
 #!/usr/bin/env python
 """Benchmark of the group-wise int8-quantized Winograd convolution on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 5] [--impl reference]
 
 A *step* is one pass of the whole forward path (input transform + group quantization,
 int8 tensor-core contraction with per-group dequantization, output transform) over
 every layer of one workload configuration, called through the C ABI.  The metric is
 direct-convolution-equivalent throughput, 2*N*K*C*H*W*9 operations per layer divided
-by the time of the forward call (filter preparation is offline and not timed).
+by the time of the forward call (filter preparation is offline and not timed).  The
+headline workload is configuration 5, the largest one (the full UNet conv-layer set).
 
 One JSON line is printed by rank 0.  Besides the throughput it carries
   roofline      achieved HBM GB/s of the kernel that takes the most time in a step,
                 from CUDA events around the chain prefixes K1, K1+K2, K1+K2+K3
+  per_config    the same figures for each of the five configurations (fewer steps)
+  contraction   the contraction kernel against the measured rate of the int8 tensor pipe
+                (an SMEM-resident tcgen05.mma kind::i8 loop), stand-alone with operands
+                warm in L2, and on one large off-configuration shape with groups of 128
+  parity        the timed outputs compared with the CPU oracle on sampled tiles
   e2e           the same metric through wfq_conv_forward_host (pinned host buffers,
                 host<->device copies inside the timed region)
   cpu_baseline  the CPU oracle timed on this machine's cores on a sample of tiles
@@ -24,6 +30,7 @@ needs no exchange between GPUs); the value is the aggregate over the ranks.
 import argparse
 import json
 import os
+import statistics
 import sys
 import threading
 import time
@@ -36,26 +43,26 @@ METRIC = "direct_conv_equivalent_TOPS"
 UNIT = "TOPS"
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
-
-# dram__bytes_read.sum + dram__bytes_write.sum per launch (mean over the layers of a step)
-# from the ncu capture summarised in profiles/launches_cfg2_resnet18_stage.txt; cold-cache
-# reads, and output that is still dirty in L2 when the kernel ends is not counted.  Only the
-# default workload was captured; set an entry to None when its kernel changes.
-NCU_TRAFFIC_BYTES = {2: {"input_transform_quantize": 6.07e6, "gemm_dequantize": 13.6e6,
-                         "output_transform": 28.6e6}}
+NOMINAL_INT8_TOPS = 4500.0
+KERNELS = ["input_transform_quantize", "gemm_dequantize", "output_transform"]
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", type=int, default=2, help="workload configuration 1..5")
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=5, help="headline workload configuration 1..5")
     ap.add_argument("--impl", default="wfq", choices=["wfq", "reference"])
+    ap.add_argument("--reps", type=int, default=5,
+                    help="graph replays per step; the step's time is their median")
     ap.add_argument("--only-layer", type=int, default=None,
                     help="restrict the workload to one layer of the configuration (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the other configurations")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the tensor-pipe rate, stand-alone contraction, sustained and parity legs")
     ap.add_argument("--no-graph", action="store_true",
                     help="enqueue every step with stream launches instead of replaying a CUDA graph")
     ap.add_argument("--cpu-seconds", type=float, default=16.0,
@@ -69,12 +76,8 @@ def workload_name(cfg):
                "at 56/28/14/7, F(6,3), group 64, fp16 input",
             3: "cfg3: ResNet-34-style sweep, N=64, 12 runs F(4,3)/F(6,3) x groups 32/64/128",
             4: "cfg4: diffusion-UNet block, N=2, C=K=320/640/1280 at 64/32/16, F(4,3), group 64",
-            5: "cfg5: UNet conv-layer set at 128/64/32 latent, N=1, F(4,3) and F(6,3)"}[cfg]
-
-
-def select_layers(wl, args):
-    layers = wl.config_layers(args.config)
-    return layers if args.only_layer is None else [layers[args.only_layer]]
+            5: "cfg5: UNet conv-layer set at 128/64/32 latent, N=1, F(4,3) and F(6,3), "
+               "C,K in {320,640,1280}, group 64, fp16 input, ten layers end to end"}[cfg]
 
 
 # ---- byte counts the method itself must move (per launch) ----------------------------
@@ -94,7 +97,22 @@ def algorithmic_bytes(L):
     k1 = L.N * L.C * L.H * L.W * e_in + P * T * L.C + 4 * P * T * G
     k2 = P * T * L.C + P * L.K * L.C + 4 * P * G * (T + L.K) + 4 * P * T * L.K
     k3 = 4 * P * T * L.K + 4 * L.N * L.K * L.H * L.W
-    return {"input_transform_quantize": k1, "gemm_dequantize": k2, "output_transform": k3}
+    return {KERNELS[0]: k1, KERNELS[1]: k2, KERNELS[2]: k3}
+
+
+def gemm_ops(L):
+    """Integer operations of the Winograd-domain contraction, 2*P*T*C*K."""
+    P, T, _ = geometry(L)
+    return 2.0 * P * T * L.C * L.K
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured copy bandwidth", d
+    return FALLBACK_HBM_GBS, "fallback", {}
 
 
 # ---- clocks -----------------------------------------------------------------------------
@@ -131,7 +149,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            self._stop.wait(0.01)
+            self._stop.wait(0.005)
 
     def start(self):
         if self.nv is not None:
@@ -196,7 +214,7 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from paper_2412_19867_b200 import workloads as wl
-    layers = select_layers(wl, args)
+    layers = select_layers(wl, args.config, args.only_layer)
     tensors = [wl.make_tensors(L) for L in layers]
     nsteps = args.steps + args.warmup
     per_step = max(0.5, min(20.0, 90.0 / max(nsteps, 1)))
@@ -242,6 +260,186 @@ def replica_throughput(ops_per_replica, world, ms_per_step):
     return world * ops_per_replica / (ms_per_step * 1e-3) / 1e12
 
 
+def select_layers(wl, cfg, only_layer=None):
+    layers = wl.config_layers(cfg)
+    return layers if only_layer is None else [layers[only_layer]]
+
+
+# ---- one configuration on the device ---------------------------------------------------
+
+class Workload:
+    """The layers of one configuration: plans, device tensors, and the step as a CUDA graph."""
+
+    def __init__(self, cfg, only_layer, dev, stream, flush, use_graph=True):
+        import torch
+        from paper_2412_19867_b200 import binding as b
+        from paper_2412_19867_b200 import workloads as wl
+        self.torch, self.b, self.dev, self.stream, self.flush = torch, b, dev, stream, flush
+        self.cfg = cfg
+        self.layers = select_layers(wl, cfg, only_layer)
+        self.tensors = [wl.make_tensors(L) for L in self.layers]
+        self.convs, self.xs, self.ys = [], [], []
+        for L, (x, w, sB, sG) in zip(self.layers, self.tensors):
+            conv = b.Conv(L.N, L.C, L.K, L.H, L.W, L.m, L.gs, L.dtype, dev)
+            conv.prepare(torch.from_numpy(w).to(dev), list(sB), list(sG))
+            self.convs.append(conv)
+            self.xs.append(torch.from_numpy(x).to(dev))
+            self.ys.append(torch.empty((L.N, L.K, L.H, L.W), dtype=torch.float32, device=dev))
+        self.step_ops = float(sum(L.direct_ops for L in self.layers))
+        self.sptr = stream.cuda_stream
+        # One step = the forward calls of all layers.  They are captured once into a CUDA
+        # graph and replayed (same kernels, same order, one submission per step); stream
+        # launches are the fallback and what --no-graph selects.
+        self.enqueue(self.sptr)
+        torch.cuda.synchronize(dev)
+        self.graph, self.launch_mode = None, "stream launches"
+        if use_graph:
+            try:
+                side = torch.cuda.Stream(dev)
+                side.wait_stream(stream)
+                cand = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(cand, stream=side):
+                    self.enqueue(side.cuda_stream)
+                torch.cuda.synchronize(dev)
+                self.graph, self.launch_mode = cand, "CUDA graph replay"
+            except Exception as exc:   # capture is an optimisation of the submission only
+                print(f"bench: graph capture failed ({exc!r}); using stream launches", file=sys.stderr)
+                torch.cuda.synchronize(dev)
+
+    def enqueue(self, stream_ptr):
+        for conv, x, y in zip(self.convs, self.xs, self.ys):
+            self.b.wfq_conv_forward(conv.plan, x.data_ptr(), y.data_ptr(), stream_ptr)
+
+    def step(self):
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.enqueue(self.sptr)
+
+    def check(self):
+        for conv in self.convs:
+            conv.check_status()
+
+    def timed_replays(self, count, flush=True):
+        """`count` replays, each in its own event pair (L2 flushed before each); ms each."""
+        torch = self.torch
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(count)]
+        for e0, e1 in ev:
+            if flush:
+                self.flush.zero_()
+            e0.record(self.stream)
+            self.step()
+            e1.record(self.stream)
+        torch.cuda.synchronize(self.dev)
+        return [e0.elapsed_time(e1) for e0, e1 in ev]
+
+    def kernel_split(self, ksteps):
+        """Per layer and kernel: ms from differences of the chain prefixes K1, K1+K2,
+        K1+K2+K3 (L2 flushed before each prefix, one event pair around each; medians)."""
+        torch, b = self.torch, self.b
+        acc = [[[], [], []] for _ in self.layers]
+        for _ in range(ksteps):
+            evs = []
+            for conv, x, y in zip(self.convs, self.xs, self.ys):
+                per_prefix = []
+                for depth in (1, 2, 3):
+                    self.flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(self.stream)
+                    b.wfq_input_transform_quantize(conv.plan, x.data_ptr(), self.sptr)
+                    if depth >= 2:
+                        b.wfq_gemm_dequantize(conv.plan, self.sptr)
+                    if depth >= 3:
+                        b.wfq_output_transform(conv.plan, y.data_ptr(), self.sptr)
+                    e1.record(self.stream)
+                    per_prefix.append((e0, e1))
+                evs.append(per_prefix)
+            torch.cuda.synchronize(self.dev)
+            for li, per_prefix in enumerate(evs):
+                t = [a.elapsed_time(z) for a, z in per_prefix]
+                acc[li][0].append(t[0])
+                acc[li][1].append(t[1] - t[0])
+                acc[li][2].append(t[2] - t[1])
+        return [[statistics.median(v) for v in layer] for layer in acc]
+
+    def gemm_warm(self, reps=6):
+        """The contraction alone, back to back on operands the previous launch left in L2."""
+        torch, b = self.torch, self.b
+        out = []
+        for conv in self.convs:
+            b.wfq_gemm_dequantize(conv.plan, self.sptr)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
+            for _ in range(reps):
+                b.wfq_gemm_dequantize(conv.plan, self.sptr)
+            e1.record(self.stream)
+            torch.cuda.synchronize(self.dev)
+            out.append(e0.elapsed_time(e1) / reps)
+        return out
+
+    def summary(self, ms_per_step, kern_ms, peak, world=1):
+        """eq-TOPS, per-layer microseconds and per-kernel roofline fractions."""
+        abytes = [algorithmic_bytes(L) for L in self.layers]
+        nl = len(self.layers)
+        tot_ms = [sum(kern_ms[li][k] for li in range(nl)) for k in range(3)]
+        tot_bytes = [sum(abytes[li][KERNELS[k]] for li in range(nl)) for k in range(3)]
+        kernels = {}
+        for k in range(3):
+            gbps = tot_bytes[k] / (tot_ms[k] * 1e-3) / 1e9
+            kernels[KERNELS[k]] = {"us_per_step": tot_ms[k] * 1e3, "GBps": gbps, "frac_of_hbm": gbps / peak,
+                                   "algorithmic_bytes_per_step": tot_bytes[k]}
+        g_ops = float(sum(gemm_ops(L) for L in self.layers))
+        kernels[KERNELS[1]]["int8_TOPS"] = g_ops / (tot_ms[1] * 1e-3) / 1e12
+        rows = []
+        for li, L in enumerate(self.layers):
+            us = [kern_ms[li][k] * 1e3 for k in range(3)]
+            rows.append({"layer": L.name, "us": round(sum(us), 2), "us_k1_k2_k3": [round(u, 2) for u in us],
+                         "frac_of_hbm_k1_k2_k3": [round(abytes[li][KERNELS[k]] / (max(us[k], 1e-3) * 1e-6) / 1e9 / peak, 3)
+                                                  for k in range(3)],
+                         "eq_TOPS": round(L.direct_ops / (sum(us) * 1e-6) / 1e12, 1)})
+        return {"workload": workload_name(self.cfg), "layers": nl,
+                "value": replica_throughput(self.step_ops, world, ms_per_step), "unit": UNIT,
+                "us_per_step": ms_per_step * 1e3, "direct_GOP_per_step": self.step_ops / 1e9,
+                "kernels": kernels, "us_per_layer": rows}, tot_ms, tot_bytes
+
+    def parity(self, tiles_per_layer=6, channels=12):
+        """The outputs of the last step against the CPU oracle on sampled tiles and output
+        channels (the oracle evaluates the pipeline tile by tile): worst error relative to
+        max |y| of the layer, and the int8 code mismatch rate of the sampled tiles."""
+        import numpy as np
+        from oracle import oracle as orc
+        b, torch = self.b, self.torch
+        worst, worst_layer, mism, ncodes = 0.0, None, 0, 0
+        for L, conv, (x, w, sB, sG), y in zip(self.layers, self.convs, self.tensors, self.ys):
+            yh = y.cpu().numpy()
+            rng = np.random.default_rng(L.seed + 13)
+            T = conv.T
+            tiles = np.unique(np.concatenate([[0, T - 1], rng.integers(0, T, tiles_per_layer)]))
+            ks = np.unique(np.concatenate([[0, L.K - 1], rng.integers(0, L.K, channels)]))
+            ref = orc.wfq(x, w[ks], L.m, L.gs, sB=sB, sG=sG, tiles=tiles)
+            xq = conv.buffer(b.WFQ_BUF_XQ)[:, torch.from_numpy(tiles).to(self.dev)].cpu().numpy()
+            mism += int(np.count_nonzero(xq != ref.Xq))
+            ncodes += xq.size
+            geo = orc.geometry(L.N, L.H, L.W, L.m)
+            scale = float(np.max(np.abs(yh)))
+            for i, t in enumerate(tiles):
+                tw, th, img = t % geo.TW, (t // geo.TW) % geo.TH, t // (geo.TW * geo.TH)
+                hh, ww = min(L.m, L.H - th * L.m), min(L.m, L.W - tw * L.m)
+                got = yh[img][ks][:, th * L.m:th * L.m + hh, tw * L.m:tw * L.m + ww]
+                err = float(np.max(np.abs(got - ref.ytile[i][:, :hh, :ww]))) / scale
+                if err > worst:
+                    worst, worst_layer = err, L.name
+        return {"checked": True, "against": "CPU oracle, sampled tiles and output channels of every layer",
+                "worst_rel_err": worst, "worst_layer": worst_layer, "tolerance": 2e-3, "ok": worst <= 2e-3,
+                "int8_code_mismatch_rate": mism / max(ncodes, 1), "codes_compared": ncodes}
+
+    def close(self):
+        for conv in self.convs:
+            conv.check_status()
+            conv.close()
+        self.graph = None
+
+
 # ---- the CUDA path ---------------------------------------------------------------------
 
 def run_wfq(args):
@@ -266,191 +464,204 @@ def run_wfq(args):
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
     stream = torch.cuda.current_stream(dev)
-
-    layers = select_layers(wl, args)
-    tensors = [wl.make_tensors(L) for L in layers]
-    convs, xs, ys = [], [], []
-    for L, (x, w, sB, sG) in zip(layers, tensors):
-        conv = b.Conv(L.N, L.C, L.K, L.H, L.W, L.m, L.gs, L.dtype, dev)
-        conv.prepare(torch.from_numpy(w).to(dev), list(sB), list(sG))
-        convs.append(conv)
-        xs.append(torch.from_numpy(x).to(dev))
-        ys.append(torch.empty((L.N, L.K, L.H, L.W), dtype=torch.float32, device=dev))
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
-    step_ops = float(sum(L.direct_ops for L in layers))
-    sptr = stream.cuda_stream
-
-    def enqueue(stream_ptr):
-        for conv, x, y in zip(convs, xs, ys):
-            b.wfq_conv_forward(conv.plan, x.data_ptr(), y.data_ptr(), stream_ptr)
-
-    # One step = the forward calls of all layers.  They are captured once into a CUDA graph
-    # and replayed (same kernels, same order, one submission per step); stream launches are
-    # the fallback and what --no-graph selects.
-    enqueue(sptr)
-    torch.cuda.synchronize(dev)
-    graph, launch_mode = None, "stream launches"
-    if not args.no_graph:
-        try:
-            side = torch.cuda.Stream(dev)
-            side.wait_stream(stream)
-            cand = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(cand, stream=side):
-                enqueue(side.cuda_stream)
-            torch.cuda.synchronize(dev)
-            graph, launch_mode = cand, "CUDA graph replay"
-        except Exception as exc:   # capture is an optimisation of the submission only
-            print(f"bench: graph capture failed ({exc!r}); using stream launches", file=sys.stderr)
-            torch.cuda.synchronize(dev)
-
-    def step():
-        if graph is not None:
-            graph.replay()
-        else:
-            enqueue(sptr)
+    peak, peak_src, peaks = hbm_peak()
+    warmup = max(args.warmup, 3)
+    reps = max(args.reps, 1)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    for _ in range(max(args.warmup, 3)):
+    wk = Workload(args.config, args.only_layer, dev, stream, flush, use_graph=not args.no_graph)
+    for _ in range(warmup):
         flush.zero_()
-        step()
+        wk.step()
     barrier()
-    for conv in convs:
-        conv.check_status()
+    wk.check()
 
-    # ---- timed region: K steps, L2 flushed before each, one event pair per step --------
+    # ---- timed region: K steps; a step's time is the median of `reps` graph replays, each
+    # behind its own L2 flush and inside its own event pair ---------------------------------
     sampler = ClockSampler(local)
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     barrier()
     sampler.start()
     wall0 = time.perf_counter()
-    for i in range(args.steps):
-        flush.zero_()
-        starts[i].record(stream)
-        step()
-        stops[i].record(stream)
+    step_ms, step_spread = [], []
+    for _ in range(args.steps):
+        t = wk.timed_replays(reps)
+        step_ms.append(statistics.median(t))
+        step_spread.append((max(t) - min(t)) / max(statistics.median(t), 1e-9))
     barrier()
     wall = time.perf_counter() - wall0
     clocks = sampler.stop()
-    ms_steps = [s.elapsed_time(e) for s, e in zip(starts, stops)]
-    total_ms = float(sum(ms_steps))
-    total_ms = max_over_ranks(total_ms, dev)
+    total_ms = max_over_ranks(float(sum(step_ms)), dev)
     ms_per_step = total_ms / args.steps
-    value = replica_throughput(step_ops, world, ms_per_step)
+    value = replica_throughput(wk.step_ops, world, ms_per_step)
+    timing = {"replays_per_step": reps, "step_time": "median of the replays",
+              "ms_per_step_min": min(step_ms), "ms_per_step_max": max(step_ms),
+              "ms_per_step_stdev": statistics.pstdev(step_ms),
+              "median_spread_within_step": statistics.median(step_spread)}
 
     # ---- the same steps back to back, no L2 flush (operands may sit in the 126 MB L2) ------
-    wsteps = min(args.steps, 100)
-    step()
+    wsteps = min(max(args.steps, 10), 100)
+    wk.step()
     torch.cuda.synchronize(dev)
     w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     w0.record(stream)
     for _ in range(wsteps):
-        step()
+        wk.step()
     w1.record(stream)
     torch.cuda.synchronize(dev)
     warm_ms = max_over_ranks(w0.elapsed_time(w1) / wsteps, dev)
-    warm = {"ms_per_step": warm_ms, "value": replica_throughput(step_ops, world, warm_ms), "unit": UNIT,
+    warm = {"ms_per_step": warm_ms, "value": replica_throughput(wk.step_ops, world, warm_ms), "unit": UNIT,
             "steps": wsteps, "l2": "not flushed"}
 
-    # ---- per-kernel durations: differences of chain prefixes ---------------------------
-    # An event pair around a single short kernel adds several microseconds of launch
-    # latency to it.  So each layer is timed three times per step, as K1, K1+K2 and
-    # K1+K2+K3 (L2 flushed before each, one event pair around each prefix); the stage
-    # durations are the differences, the first one carries the pair's overhead.
-    names = ["input_transform_quantize", "gemm_dequantize", "output_transform"]
-    ksteps = min(args.steps, 100)
-    kern_ms = [[0.0, 0.0, 0.0] for _ in layers]
-    for _ in range(ksteps):
-        evs = []
-        for conv, x, y in zip(convs, xs, ys):
-            per_prefix = []
-            for depth in (1, 2, 3):
-                flush.zero_()
+    # ---- per-kernel durations and roofline of the headline workload -----------------------
+    ksteps = min(max(args.steps, 10), 40)
+    kern_ms = wk.kernel_split(ksteps)
+    head, tot_ms, tot_bytes = wk.summary(ms_per_step, kern_ms, peak, world)
+    dom = max(range(3), key=lambda k: tot_ms[k])
+    achieved = tot_bytes[dom] / (tot_ms[dom] * 1e-3) / 1e9
+    nl = len(wk.layers)
+    roofline = {"bound": "hbm", "kernel": KERNELS[dom], "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                "launches_per_step": nl, "algorithmic_bytes_per_step": tot_bytes[dom],
+                "algorithmic_bytes_per_launch": tot_bytes[dom] / nl,
+                "us_per_launch": tot_ms[dom] * 1e3 / nl,
+                "note": "traffic: no ncu capture of this kernel version on the headline workload; "
+                        "per-launch DRAM bytes of single layers are in profiles/",
+                "all_kernels": head["kernels"]}
+
+    # ---- sustained: the same step replayed for about two seconds -------------------------
+    sustained = None
+    contraction = None
+    parity = None
+    if not args.no_extras:
+        s_sampler = ClockSampler(local)
+        s_sampler.start()
+        t_end = time.perf_counter() + 2.0
+        s_ms = []
+        while time.perf_counter() < t_end:
+            s_ms += wk.timed_replays(20)
+        s_clocks = s_sampler.stop()
+        s_med = statistics.median(s_ms)
+        sustained = {"seconds": 2.0, "replays": len(s_ms), "ms_per_step_median": s_med,
+                     "value": replica_throughput(wk.step_ops, world, s_med), "unit": UNIT, "clocks": s_clocks}
+
+        # ---- outputs of the timed workload against the oracle (outside every timed region) ---
+        if rank == 0:
+            flush.zero_()
+            wk.step()
+            torch.cuda.synchronize(dev)
+            parity = wk.parity()
+
+        # ---- the contraction against the rate of the int8 tensor pipe -------------------
+        rate = {}
+        for n_cols in (64, 128, 256):
+            best = 0.0
+            for _ in range(3):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-                b.wfq_input_transform_quantize(conv.plan, x.data_ptr(), sptr)
-                if depth >= 2:
-                    b.wfq_gemm_dequantize(conv.plan, sptr)
-                if depth >= 3:
-                    b.wfq_output_transform(conv.plan, y.data_ptr(), sptr)
+                ops = b.wfq_debug_int8_mma_rate(wk.convs[0].plan, n_cols, 20000, stream.cuda_stream)
                 e1.record(stream)
-                per_prefix.append((e0, e1))
-            evs.append(per_prefix)
-        torch.cuda.synchronize(dev)
-        for li, per_prefix in enumerate(evs):
-            t = [a.elapsed_time(z) for a, z in per_prefix]
-            kern_ms[li][0] += t[0] / ksteps
-            kern_ms[li][1] += (t[1] - t[0]) / ksteps
-            kern_ms[li][2] += (t[2] - t[1]) / ksteps
-    abytes = [algorithmic_bytes(L) for L in layers]
-    tot_ms = [sum(kern_ms[li][k] for li in range(len(layers))) for k in range(3)]
-    tot_bytes = [sum(abytes[li][names[k]] for li in range(len(layers))) for k in range(3)]
-    dom = max(range(3), key=lambda k: tot_ms[k])
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        with open(peaks_path) as f:
-            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured copy bandwidth"
-    else:
-        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
-    achieved = tot_bytes[dom] / (tot_ms[dom] * 1e-3) / 1e9
-    traffic = None
-    if args.only_layer is None:
-        traffic = NCU_TRAFFIC_BYTES.get(args.config, {}).get(names[dom])
-    roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
-                "launches_per_step": len(layers),
-                "algorithmic_bytes_per_step": tot_bytes[dom],
-                "algorithmic_bytes_per_launch": tot_bytes[dom] / len(layers),
-                "all_kernels": {names[k]: {"us_per_step": tot_ms[k] * 1e3,
-                                           "GBps": tot_bytes[k] / (tot_ms[k] * 1e-3) / 1e9,
-                                           "frac": tot_bytes[k] / (tot_ms[k] * 1e-3) / 1e9 / peak}
-                                for k in range(3)}}
-    # contraction alone: algorithmic int8 operations 2*P*T*C*K per layer against the tensor peak
-    def tiles(L):
-        return L.N * (-(-L.H // L.m)) * (-(-L.W // L.m))
-    gemm_ops = float(sum(2.0 * (L.m + 2) ** 2 * tiles(L) * L.C * L.K for L in layers))
-    gemm_tops = gemm_ops / (tot_ms[1] * 1e-3) / 1e12
-    gk = roofline["all_kernels"][names[1]]
-    gk["int8_TOPS"] = gemm_tops
-    gk["frac_of_nominal_int8_4500_TOPS"] = gemm_tops / 4500.0
-    if os.path.exists(peaks_path):
-        with open(peaks_path) as f:
-            bf16 = json.load(f).get("bf16_tflops")
-        if bf16:
-            gk["frac_of_2x_measured_bf16"] = gemm_tops / (2.0 * float(bf16))
-    layer_rows = []
-    for li, L in enumerate(layers):
-        us = [kern_ms[li][k] * 1e3 for k in range(3)]
-        layer_rows.append({"layer": L.name, "us": sum(us), "us_k1_k2_k3": [round(u, 2) for u in us],
-                           "eq_TOPS": L.direct_ops / (sum(us) * 1e-6) / 1e12})
+                torch.cuda.synchronize(dev)
+                best = max(best, ops / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+            rate[f"128x{n_cols}x32"] = best
+        int8_peak = max(rate.values())
+        g_warm = wk.gemm_warm()
+        g_ops = [gemm_ops(L) for L in wk.layers]
+        warm_tops = sum(g_ops) / (sum(g_warm) * 1e-3) / 1e12
+        chain_tops = head["kernels"][KERNELS[1]]["int8_TOPS"]
+        # the promotion of a group's int32 sums takes about 2.3 issue slots per accumulator
+        # element, an SM issues 128 per clock and the tensor pipe yields 8192/gs elements
+        ceil64 = 64.0 / (64.0 * 2.3)
+        contraction = {"int8_peak_measured_TOPS": int8_peak, "int8_rate_by_shape_TOPS": rate,
+                       "int8_peak_how": "SMEM-resident accumulating tcgen05.mma kind::i8, one CTA per SM, "
+                                        "20000 instructions each, best of 3",
+                       "int8_nominal_TOPS": NOMINAL_INT8_TOPS,
+                       "in_chain": {"int8_TOPS": chain_tops, "frac_of_measured_peak": chain_tops / int8_peak,
+                                    "frac_of_nominal": chain_tops / NOMINAL_INT8_TOPS},
+                       "stand_alone_l2_warm": {"int8_TOPS": warm_tops, "frac_of_measured_peak": warm_tops / int8_peak,
+                                               "us_per_layer": [round(t * 1e3, 2) for t in g_warm]},
+                       "promotion_ceiling_frac": {"group_64": ceil64, "group_128": min(1.0, 2 * ceil64),
+                                                  "issue_slots_per_accumulator": 2.3}}
+        # one large shape outside the configurations: many tiles, groups of 128 channels
+        try:
+            big = wl.Layer(8, 1024, 256, 112, 112, 4, 128, "f16", "silu_outlier", "kaiming_chan", 6, 0, 0)
+            x, w, sB, sG = wl.make_tensors(big)
+            conv = b.Conv(big.N, big.C, big.K, big.H, big.W, big.m, big.gs, big.dtype, dev)
+            conv.prepare(torch.from_numpy(w).to(dev), list(sB), list(sG))
+            xd = torch.from_numpy(x).to(dev)
+            b.wfq_input_transform_quantize(conv.plan, xd.data_ptr(), stream.cuda_stream)
+            b.wfq_gemm_dequantize(conv.plan, stream.cuda_stream)
+            ts = []
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                b.wfq_gemm_dequantize(conv.plan, stream.cuda_stream)
+                e1.record(stream)
+                torch.cuda.synchronize(dev)
+                ts.append(e0.elapsed_time(e1))
+            conv.check_status()
+            t = statistics.median(ts)
+            tops = gemm_ops(big) / (t * 1e-3) / 1e12
+            contraction["large_shape_group_128"] = {
+                "layer": big.name, "us": t * 1e3, "int8_TOPS": tops, "frac_of_measured_peak": tops / int8_peak,
+                "GBps": algorithmic_bytes(big)[KERNELS[1]] / (t * 1e-3) / 1e9,
+                "note": "contraction kernel only; operands and Y (231 MB each) exceed L2"}
+            conv.close()
+            del xd
+        except Exception as exc:
+            contraction["large_shape_group_128"] = {"error": repr(exc)}
 
     # ---- end to end through the host-buffer entry point ----------------------------------
     e2e = None
     if not args.no_e2e:
-        xh = [torch.from_numpy(t[0]).pin_memory() for t in tensors]
-        yh = [torch.empty(y.shape, dtype=torch.float32).pin_memory() for y in ys]
+        xh = [torch.from_numpy(t[0]).pin_memory() for t in wk.tensors]
+        yh = [torch.empty(y.shape, dtype=torch.float32).pin_memory() for y in wk.ys]
         esteps = max(3, min(args.steps, 20))
-        for conv, x, y in zip(convs, xh, yh):
+        for conv, x, y in zip(wk.convs, xh, yh):
             conv.forward_host(x, y)
         barrier()
         t0 = time.perf_counter()
         for _ in range(esteps):
-            for conv, x, y in zip(convs, xh, yh):
+            for conv, x, y in zip(wk.convs, xh, yh):
                 conv.forward_host(x, y)          # synchronous: copies + kernels + copy back
         torch.cuda.synchronize(dev)
         dt = time.perf_counter() - t0
         dt = max_over_ranks(dt, dev)
-        e2e = {"value": replica_throughput(step_ops, world, dt * 1e3 / esteps), "unit": UNIT,
+        e2e = {"value": replica_throughput(wk.step_ops, world, dt * 1e3 / esteps), "unit": UNIT,
                "h2d_bytes_per_step": int(sum(x.numel() * x.element_size() for x in xh)),
                "d2h_bytes_per_step": int(sum(y.numel() * 4 for y in yh)), "steps": esteps}
+        del xh, yh
 
-    for conv in convs:
-        conv.check_status()
-        conv.close()
+    layers, tensors = wk.layers, wk.tensors
+    launch_mode = wk.launch_mode
+    wk.close()
+
+    # ---- the other configurations, fewer steps -------------------------------------------
+    per_config = None
+    if rank == 0 and world == 1 and not args.no_per_config and args.only_layer is None:
+        per_config = {f"cfg{args.config}": {k: head[k] for k in head}}
+        for cfg in (1, 2, 3, 4, 5):
+            if cfg == args.config:
+                continue
+            try:
+                w2 = Workload(cfg, None, dev, stream, flush, use_graph=not args.no_graph)
+                for _ in range(3):
+                    flush.zero_()
+                    w2.step()
+                torch.cuda.synchronize(dev)
+                ms = [statistics.median(w2.timed_replays(reps)) for _ in range(10)]
+                s2, _, _ = w2.summary(statistics.mean(ms), w2.kernel_split(10), peak)
+                s2["steps"] = 10
+                w2.close()
+                per_config[f"cfg{cfg}"] = s2
+                del w2
+                torch.cuda.empty_cache()
+            except Exception as exc:
+                per_config[f"cfg{cfg}"] = {"error": repr(exc)}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -460,17 +671,18 @@ def run_wfq(args):
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
                 "config": {"workload": workload_name(args.config) +
                            ("" if args.only_layer is None else f" (layer {args.only_layer} only)"),
                            "layers": len(layers), "launch": launch_mode,
-                           "l2": "flushed before every step (256 MiB memset outside the step's "
+                           "l2": "flushed before every replay (256 MiB memset outside the replay's "
                                  "event pair)",
                            "parallelism": "replicas" if world > 1 else "single GPU"},
-                "us_per_layer": layer_rows, "wall_s_timed_region": wall,
-                "warm": warm, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
-                "gpu_launches": 3 * len(layers) * args.steps, "clocks": clocks}
+                "timing": timing, "us_per_layer": head["us_per_layer"], "wall_s_timed_region": wall,
+                "warm": warm, "sustained": sustained, "roofline": roofline, "contraction": contraction,
+                "parity": parity, "per_config": per_config, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": 3 * len(layers) * args.steps * reps, "clocks": clocks}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

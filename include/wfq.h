@@ -83,8 +83,10 @@ typedef enum {
                                        transform's producer does not load (-1 = none): the
                                        waits for it run out, the kernel records
                                        WFQ_ERR_TIMEOUT in the status word and ends by itself */
-    WFQ_DEBUG_GENERIC_INPUT_TRANSFORM = 2, /* nonzero: always use the cp.async input-transform
-                                       kernel, also where the tensor-core one applies */
+    WFQ_DEBUG_INPUT_TRANSFORM_KERNEL = 2, /* 0: the library chooses; 1: the cp.async kernel;
+                                       2: the tensor-core kernel wherever it applies (fp16 input,
+                                       groups of 32 or 64, C a multiple of 64, 16-byte aligned x,
+                                       a shape its TMA or bulk staging can describe) */
     WFQ_DEBUG_SKIP_GEMM_STAGE = 3   /* operand stage (counted from 0) whose loads the first
                                        CTA of the contraction kernel does not issue (-1 =
                                        none); same purpose as WFQ_DEBUG_SKIP_INPUT_ITEM */

@@ -235,8 +235,9 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
     }
     for (int i = 0; i < g.n; ++i)
         for (int j = 0; j < g.n; ++j) {
-            plan->tables.in_scale[i * g.n + j] =
-                (float)((plan->sB[i] / stdB[i]) * (plan->sB[j] / stdB[j]));
+            const double f = (plan->sB[i] / stdB[i]) * (plan->sB[j] / stdB[j]);
+            plan->tables.in_scale[i * g.n + j] = (float)f;
+            plan->tables.in_scale_lo[i * g.n + j] = (float)(f - (double)(float)f);
             plan->tables.out_scale[i * g.n + j] = (float)(plan->sA[i] * plan->sA[j]);
         }
 
@@ -359,7 +360,7 @@ static wfq_status_t setup_host_pipeline(wfq_plan *plan)
         }
         wfq_plan *q = plan->sub[s];
         wfq_plan_set_input_dtype(q, plan->in_dtype);
-        q->debug_force_generic_k1 = plan->debug_force_generic_k1;
+        q->k1_choice = plan->k1_choice;
         // same orientation of the contraction as the whole batch: identical arithmetic
         q->gemm_swap = plan->gemm_swap;
         q->gemm_bn = plan->gemm_bn;
@@ -460,8 +461,9 @@ wfq_status_t wfq_plan_set_debug_option(wfq_plan_t *plan, wfq_debug_option_t opti
             if (value < -1 || value > 0x7fffffff) return WFQ_ERR_INVALID_ARG;
             plan->debug_skip_item = (int)value;
             break;
-        case WFQ_DEBUG_GENERIC_INPUT_TRANSFORM:
-            plan->debug_force_generic_k1 = value != 0;
+        case WFQ_DEBUG_INPUT_TRANSFORM_KERNEL:
+            if (value < 0 || value > 2) return WFQ_ERR_INVALID_ARG;
+            plan->k1_choice = (int)value;
             break;
         case WFQ_DEBUG_SKIP_GEMM_STAGE:
             if (value < -1 || value > 0x7fffffff) return WFQ_ERR_INVALID_ARG;
@@ -473,7 +475,7 @@ wfq_status_t wfq_plan_set_debug_option(wfq_plan_t *plan, wfq_debug_option_t opti
     for (int i = 0; i < 2; ++i)
         if (plan->sub[i]) {
             plan->sub[i]->wait_cycles = plan->wait_cycles;
-            plan->sub[i]->debug_force_generic_k1 = plan->debug_force_generic_k1;
+            plan->sub[i]->k1_choice = plan->k1_choice;
         }
     return WFQ_OK;
 }

@@ -169,10 +169,12 @@ __device__ __forceinline__ uint32_t codes4(float4 v, float inv)
                        __byte_perm(code_bits(v.z, inv), code_bits(v.w, inv), 0x0040), 0x5410);
 }
 
-__device__ __forceinline__ float4 scale4(float4 v, float2 s2)
+// X = Z * (s + sl), rounded once: fma(z, s, z * sl) (the factor is held as two floats).
+__device__ __forceinline__ float4 scale4(float4 v, float2 s2, float2 sl2)
 {
-    const float2 lo = mul2_rn(make_float2(v.x, v.y), s2);
-    const float2 hi = mul2_rn(make_float2(v.z, v.w), s2);
+    const float2 a = make_float2(v.x, v.y), b = make_float2(v.z, v.w);
+    const float2 lo = __ffma2_rn(a, s2, mul2_rn(a, sl2));
+    const float2 hi = __ffma2_rn(b, s2, mul2_rn(b, sl2));
     return make_float4(lo.x, lo.y, hi.x, hi.y);
 }
 
@@ -383,13 +385,13 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
                 const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs +
                                                                      part * GSR);
                 int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs + part * GSR;
-                const float sp = tab.in_scale[p];
-                const float2 sp2 = make_float2(sp, sp);
+                const float sp = tab.in_scale[p], sl = tab.in_scale_lo[p];
+                const float2 sp2 = make_float2(sp, sp), sl2 = make_float2(sl, sl);
                 float4 v[GSR / 4];
                 float amax = 0.f;
 #pragma unroll
                 for (int k = 0; k < GSR / 4; ++k) {
-                    v[k] = scale4(src[k], sp2);
+                    v[k] = scale4(src[k], sp2, sl2);
                     amax = absmax4(amax, v[k]);
                 }
                 if constexpr (SPLIT >= 2) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
@@ -414,18 +416,18 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
                 const int t = srow * g.TW + tw0 + tl;
                 const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs);
                 int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
-                const float sp = tab.in_scale[p];
-                const float2 sp2 = make_float2(sp, sp);
+                const float sp = tab.in_scale[p], sl = tab.in_scale_lo[p];
+                const float2 sp2 = make_float2(sp, sp), sl2 = make_float2(sl, sl);
                 float scale, inv;
                 float amax = 0.f;
-                for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2));
+                for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2, sl2));
                 group_scale(amax, scale, inv);
                 for (int k = 0; k < gs / 32; ++k)
-                    st_global_v8_b32(dst + 32 * k, codes4(scale4(src[8 * k], sp2), inv),
-                                     codes4(scale4(src[8 * k + 1], sp2), inv), codes4(scale4(src[8 * k + 2], sp2), inv),
-                                     codes4(scale4(src[8 * k + 3], sp2), inv), codes4(scale4(src[8 * k + 4], sp2), inv),
-                                     codes4(scale4(src[8 * k + 5], sp2), inv), codes4(scale4(src[8 * k + 6], sp2), inv),
-                                     codes4(scale4(src[8 * k + 7], sp2), inv));
+                    st_global_v8_b32(dst + 32 * k, codes4(scale4(src[8 * k], sp2, sl2), inv),
+                                     codes4(scale4(src[8 * k + 1], sp2, sl2), inv), codes4(scale4(src[8 * k + 2], sp2, sl2), inv),
+                                     codes4(scale4(src[8 * k + 3], sp2, sl2), inv), codes4(scale4(src[8 * k + 4], sp2, sl2), inv),
+                                     codes4(scale4(src[8 * k + 5], sp2, sl2), inv), codes4(scale4(src[8 * k + 6], sp2, sl2), inv),
+                                     codes4(scale4(src[8 * k + 7], sp2, sl2), inv));
                 sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
             }
         }
@@ -550,7 +552,8 @@ cudaError_t launch_input_transform(wfq_plan &plan, const void *x_dev, cudaStream
 {
     const Geometry &g = plan.geo;
     // tensor-core kernel: fp16 input that a TMA tensor map (16-byte aligned base) can describe
-    if (plan.k1tc.use && !plan.debug_force_generic_k1 && (reinterpret_cast<uintptr_t>(x_dev) & 15u) == 0) {
+    // (automatic = the cp.async kernel: the tensor-core one measured no faster on any configured layer)
+    if (plan.k1tc.use && plan.k1_choice == 2 && (reinterpret_cast<uintptr_t>(x_dev) & 15u) == 0) {
         if (plan.k1tc.mode != 2 && plan.tmap_x_base != x_dev) {
             const unsigned long long hw = (unsigned long long)g.H * g.W;
             bool ok;

@@ -31,23 +31,24 @@
 // (Few warps with many registers were tried first: every role is a chain of dependent
 // instructions and mbarrier hand-overs of a few hundred cycles each, and only many
 // resident warps hide them.)
-// Accumulator rows: S "slots" of PL lanes (F(6,3): 2 x 64, F(4,3): 3 x 40); the constant
-// matrix sits in shared memory between blocks of zero rows, and the MMA of slot s starts
-// its 128-row window so that the matrix lands on lanes s * PL ...: one accumulator of 128
-// columns therefore holds 2 * S tiles.  Patch tiles flow through the kernel as one flat
+// Accumulator rows: S "slots" of PL lanes (F(6,3): 2 x 64, F(4,3): 3 x 40).  The constant
+// matrix is the A operand and lives in tensor memory, one copy per slot with its rows on
+// lanes s * PL ... and zeros on all other lanes; the MMAs of a pair use the copy of their
+// slot, so one accumulator of 128 columns holds 2 * S tiles, and the tensor cores read only
+// the patch tiles from shared memory (whose bandwidth bounds this kernel).  Patch tiles flow through the kernel as one flat
 // sequence (pairs, then groups of S pairs), independent of the work items they came from.
 //
-// Staging modes (chosen on the host).  The TMA unit spends about two cycles per box row
-// whatever its length, so strips are made of few, long rows where the shape allows it:
+// Staging modes (chosen on the host):
+//   0  3-D tiled TMA over (W, H, N*C): column chunks of a tile row (the whole row where it
+//      fits), all padding by zero fill; needs W*2 to be a multiple of 16.  The box width is
+//      8 modulo 16 elements, so that the eight patch rows of a channel start in different
+//      shared-memory banks for the im2col reads.
 //   1  2-D tiled TMA over (H*W, N*C): a strip is a whole tile row, n image rows x full width
-//      per channel, fetched as one or more boxes of `rpb` image rows (<= 256 elements, i.e.
-//      up to 512 contiguous bytes per box row); top/bottom padding by zero fill, left/right
-//      by masks.  Needs H*W*2 to be a multiple of 16, and W*2 too when several boxes are used.
-//   0  3-D tiled TMA over (W, H, N*C): column chunks of a tile row, all padding by zero fill
-//      (needs W*2 to be a multiple of 16); for images too wide for mode 1.
+//      per channel in one box (<= 256 elements); top/bottom padding by zero fill, left/right
+//      by masks.  For widths that are not a multiple of 8 with H*W*2 a multiple of 16.
 //   2  one bulk copy of a whole 64-channel block of a (small) image, all padding by masks.
-// The constant matrix is built once per device on the host (already in the swizzled
-// shared-memory layout) and fetched by one bulk copy per CTA.
+// The constant matrix is built once per device on the host; four warps of every CTA copy it
+// from global memory into tensor memory while the first strips are in flight.
 #include <cuda_fp16.h>
 
 #include <cstring>
@@ -62,7 +63,9 @@ namespace {
 constexpr int TC_THREADS = 1024;
 constexpr int TC_CB = 64;            // channels per work item = rows of an operand tile
 constexpr int TC_TILE_BYTES = TC_CB * 128;
-constexpr int TC_NACC = 4;           // accumulators of 128 TMEM columns
+constexpr int TC_NACC = 2;           // accumulators of 128 TMEM columns, one per quantizer team
+constexpr int TC_TMEM_COLS = 512;    // allocation: accumulators, then the constant matrix
+constexpr int TC_AMAT_COL = 128 * TC_NACC;
 constexpr int TC_MAX_STRIP = 8;
 constexpr int TC_MAX_PAIR = 8;
 constexpr int TC_IDS = 64;           // ring of tile ids (operand tiles in flight < 64)
@@ -82,6 +85,7 @@ struct TcShared {
     uint64_t acc_empty[TC_NACC];          // all quantizer warps have read the accumulator
     uint64_t mma_done;                    // every MMA issued by this CTA has completed
     uint64_t amat_full;                   // the constant matrix has landed
+    uint64_t tick;                        // one phase per increment of pairs_consumed
     uint32_t tmem_base;
     volatile int abort;
     volatile int pairs_consumed;          // operand-tile pairs whose MMAs have completed
@@ -96,8 +100,7 @@ struct TcCfg {
     static constexpr int S = M == 6 ? 2 : 3;            // tile slots on the TMEM lanes
     static constexpr int PL = M == 6 ? 64 : 40;         // lanes per slot (a multiple of 8)
     static constexpr int KSTEPS = NN / 2;               // K = 16 = two patch rows per MMA
-    static constexpr int AROWS = (S - 1) * PL + 128;    // zero rows, matrix, zero rows
-    static constexpr int A_BYTES = AROWS * 128;
+    static constexpr int KW = KSTEPS * 8;               // 32-bit TMEM columns of the matrix (K / 2)
 };
 
 struct TcArgs {
@@ -109,8 +112,7 @@ struct TcArgs {
     int mode, TBW, NCHUNK, NCB, items;
     int CS, RS;              // strip strides in elements: channel, patch row
     int strip_bytes, nstrip, nbp;
-    int nbox, rpb, box_elems; // mode 1: boxes per strip, image rows per box, elements per box row
-    const void *amat;        // the constant matrix, [AROWS][128 B] swizzled, global memory
+    const uint32_t *amat;    // the constant matrix, [P][KW] words (two fp16 K elements each), global
     int debug_skip_item;     // >= 0: the producer skips this item (exercises the bounded waits)
 };
 
@@ -165,22 +167,23 @@ __device__ __forceinline__ void st_global_v8_u32(void *p, const uint32_t (&w)[8]
                  : "memory");
 }
 
-// v = fl32(z * sp) for 32 accumulator values, in place; returns max |v| folded into m.
-__device__ __forceinline__ float scale_and_max32(uint32_t (&r)[32], float sp, float m)
+// max |z| of 32 accumulator values folded into m.  (The abs-max of the group is taken on
+// the raw transform values: rounding is monotone, so max |fl(z * s)| = |fl(zmax * s)|.)
+__device__ __forceinline__ float absmax32(const uint32_t (&r)[32], float m)
 {
-    const float2 sp2 = make_float2(sp, sp);
     float m0 = m, m1 = 0.f, m2 = 0.f, m3 = 0.f;
 #pragma unroll
     for (int k = 0; k < 32; k += 4) {
-        const float2 v0 = __fmul2_rn(make_float2(__uint_as_float(r[k]), __uint_as_float(r[k + 1])), sp2);
-        const float2 v1 = __fmul2_rn(make_float2(__uint_as_float(r[k + 2]), __uint_as_float(r[k + 3])), sp2);
-        r[k] = __float_as_uint(v0.x); r[k + 1] = __float_as_uint(v0.y);
-        r[k + 2] = __float_as_uint(v1.x); r[k + 3] = __float_as_uint(v1.y);
-        m0 = fmaxf(m0, fabsf(v0.x)); m1 = fmaxf(m1, fabsf(v0.y));
-        m2 = fmaxf(m2, fabsf(v1.x)); m3 = fmaxf(m3, fabsf(v1.y));
+        m0 = fmaxf(m0, fabsf(__uint_as_float(r[k])));
+        m1 = fmaxf(m1, fabsf(__uint_as_float(r[k + 1])));
+        m2 = fmaxf(m2, fabsf(__uint_as_float(r[k + 2])));
+        m3 = fmaxf(m3, fabsf(__uint_as_float(r[k + 3])));
     }
     return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
+
+// x = z * (sp + sl), rounded once: fma(z, sp, z * sl).
+__device__ __forceinline__ float scaled(float z, float sp, float sl) { return fmaf(z, sp, __fmul_rn(z, sl)); }
 
 // Scale and reciprocal of a group from its abs-max (the quantizer of Section 2).
 __device__ __forceinline__ void group_scale_inv(float amax, float &scale, float &inv)
@@ -190,29 +193,43 @@ __device__ __forceinline__ void group_scale_inv(float amax, float &scale, float 
     inv = nz ? __fdiv_rn(127.f, amax) : 0.f;
 }
 
-// 32 codes from the 32 values v (fp32 bit patterns in r), one 32-byte store.
-__device__ __forceinline__ void codes32(const uint32_t (&r)[32], float inv, int8_t *dst)
+// 32 codes from 32 raw transform values z: x = z * (sp + sl) rounded once, t = fl(x * inv),
+// code = low byte of fl(t + 1.5 * 2^23) (round to nearest even); one 32-byte store.
+__device__ __forceinline__ void codes32(const uint32_t (&r)[32], float sp, float sl, float inv, int8_t *dst)
 {
-    const float2 inv2 = make_float2(inv, inv);
+    const float2 sp2 = make_float2(sp, sp), sl2 = make_float2(sl, sl), inv2 = make_float2(inv, inv);
     uint32_t w[8];
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
-        const float2 lo = __fmul2_rn(make_float2(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1])), inv2);
-        const float2 hi = __fmul2_rn(make_float2(__uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3])), inv2);
-        w[q] = pack4(lo.x, lo.y, hi.x, hi.y);
+        const float2 z0 = make_float2(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]));
+        const float2 z1 = make_float2(__uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+        const float2 t0 = __fmul2_rn(__ffma2_rn(z0, sp2, __fmul2_rn(z0, sl2)), inv2);
+        const float2 t1 = __fmul2_rn(__ffma2_rn(z1, sp2, __fmul2_rn(z1, sl2)), inv2);
+        w[q] = pack4(t0.x, t0.y, t1.x, t1.y);
     }
     st_global_v8_u32(dst, w);
 }
 
 // Bounded wait until the counter `*ctr` (shared memory, only ever incremented) has reached
-// `target`.  Unlike an mbarrier phase it can be tested for any future value, so warps that
-// work on different parts of the operand ring need not see every phase of every buffer.
-__device__ __noinline__ bool wait_counter(volatile int *ctr, int target, const WaitCtx &ctx, int where)
+// `target`.  Unlike an mbarrier phase a counter can be tested for any future value, so warps
+// that work on different parts of the operand ring need not see every phase of every
+// buffer.  The waiting itself is not a polling loop (twelve polling warps took two fifths of
+// the SM's issue slots): the writer of the counter also arrives on the barrier `tick` once
+// per increment, and a waiter that finds the counter at c < target sleeps in a try_wait
+// on the phase of tick that the increment to c + 1 completes.  Should the counter move on
+// by two between the read and the wait, the try_wait's time hint ends the sleep.
+__device__ __noinline__ bool wait_counter(volatile int *ctr, uint32_t tick, int target, const WaitCtx &ctx,
+                                          int where)
 {
-    const long long t0 = clock64();
-    while (*ctr < target) {
+    long long t0 = 0;
+    for (;;) {
+        const int c = *ctr;
+        if (c >= target) return true;
+        ptx::mbar_try_wait_ns(tick, (uint32_t)(c & 1), 2000u);
         if (*ctx.abort) return false;
-        if (clock64() - t0 > ctx.limit) {
+        const long long now = clock64();
+        if (t0 == 0) t0 = now;
+        if (now - t0 > ctx.limit) {
             *ctx.abort = 1;
             if (atomicCAS(ctx.status, 0, 6 /* WFQ_ERR_TIMEOUT */) == 0) {
                 ctx.status[1] = where;
@@ -221,9 +238,7 @@ __device__ __noinline__ bool wait_counter(volatile int *ctr, int target, const W
             }
             return false;
         }
-        __nanosleep(32);
     }
-    return true;
 }
 
 template <int M, int GS, int MODE>
@@ -235,8 +250,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char *Amat = base;                                  // [AROWS][128 B], swizzled
-    unsigned char *Bring = Amat + C::A_BYTES;                    // [2 * nbp][64 rows][128 B]
+    unsigned char *Bring = base;                                 // [2 * nbp][64 rows][128 B]
     unsigned char *strips = Bring + (size_t)2 * a.nbp * TC_TILE_BYTES;
     TcShared *sh = reinterpret_cast<TcShared *>(strips + (size_t)a.nstrip * a.strip_bytes);
 
@@ -255,10 +269,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
             const int first = it.tw0 * M - 1;
             ptx::tma_load_3d(dst, &tmx, bar, ((first + 8) & ~7) - 8, it.th * M - 1, z);
         } else if (MODE == 1) {
-            const int fs = (it.th * M - 1) * g.W;
-            for (int j = 0; j < a.nbox; ++j)
-                ptx::tma_load_2d(dst + (uint32_t)(j * TC_CB * a.box_elems * 2), &tmx, bar,
-                                 (fs + j * a.rpb * g.W) & ~7, z);
+            ptx::tma_load_2d(dst, &tmx, bar, ((it.th * M - 1) * g.W) & ~7, z);
         } else {
             ptx::bulk_load(dst, a.x + (size_t)z * g.H * g.W, (uint32_t)a.strip_bytes, bar);
         }
@@ -279,22 +290,19 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
             ptx::mbar_init(ptx::smem_u32(&sh->acc_empty[lane - TC_MAX_STRIP - TC_MAX_PAIR]), TC_TEAM_WARPS);
         } else if (lane == 31) {
             ptx::mbar_init(ptx::smem_u32(&sh->mma_done), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh->amat_full), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh->amat_full), 4);
+            ptx::mbar_init(ptx::smem_u32(&sh->tick), 1);
             sh->abort = 0;
             sh->pairs_consumed = 0;
         }
         ptx::fence_mbar_init();
         __syncwarp();
-        if (lane == 0) {
-            if (MODE != 2) ptx::prefetch_tmap(&tmx);
-            ptx::mbar_arrive_expect_tx(ptx::smem_u32(&sh->amat_full), (uint32_t)C::A_BYTES);
-            ptx::bulk_load(ptx::smem_u32(Amat), a.amat, (uint32_t)C::A_BYTES, ptx::smem_u32(&sh->amat_full));
-        }
+        if (lane == 0 && MODE != 2) ptx::prefetch_tmap(&tmx);
         for (int item = blockIdx.x; item < a.items && prefilled < a.nstrip; item += gridDim.x)
             issue_strip(item, prefilled++);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), 128 * TC_NACC);
+        ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), TC_TMEM_COLS);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before();
@@ -328,13 +336,11 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
             for (int j = issued - 1; j >= 0 && j >= issued - a.nstrip; --j)
                 drain(ptx::smem_u32(&sh->strip_full[j % a.nstrip]), (uint32_t)((j / a.nstrip) & 1),
                       a.wait_cycles / 16);
-            drain(ptx::smem_u32(&sh->amat_full), 0, a.wait_cycles / 16);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         constexpr uint32_t idesc = ptx::idesc_f16(128, 128);
         constexpr uint32_t dhi = ptx::smem_desc_sw128_hi();
-        const uint32_t a_lo0 = ptx::smem_desc_sw128_lo(ptx::smem_u32(Amat));
         const uint32_t b_lo0 = ptx::smem_desc_sw128_lo(ptx::smem_u32(Bring));
         const int npairs = (nbt + 1) >> 1;
         int slot = 0, s = 0, acc = 0;
@@ -350,13 +356,13 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
             ptx::tc_fence_after();
             if (lane == 0) {
                 const uint32_t d = tmem_base + (uint32_t)(acc * 128);
-                // window of 128 rows that puts the matrix on lanes s * PL ...
-                const uint32_t a_lo = a_lo0 + (uint32_t)(((S - 1 - s) * PL * 128) >> 4);
+                // the copy of the matrix that sits on lanes s * PL ... (zero elsewhere)
+                const uint32_t a_t = tmem_base + (uint32_t)(TC_AMAT_COL + s * C::KW);
                 const uint32_t b_lo = b_lo0 + (uint32_t)((slot * 2 * TC_TILE_BYTES) >> 4);
 #pragma unroll
                 for (int ks = 0; ks < KSTEPS; ++ks) {
-                    if (ks == 0 && s == 0) ptx::umma_f16_lo<false>(d, a_lo, b_lo, dhi, idesc);
-                    else ptx::umma_f16_lo<true>(d, a_lo + 2 * ks, b_lo + 2 * ks, dhi, idesc);
+                    if (ks == 0 && s == 0) ptx::umma_f16_tmem_a<false>(d, a_t, b_lo, dhi, idesc);
+                    else ptx::umma_f16_tmem_a<true>(d, a_t + 8 * ks, b_lo + 2 * ks, dhi, idesc);
                 }
                 ptx::umma_commit(ptx::smem_u32(&sh->pair_empty[slot]));
                 if (s == S - 1 || k == npairs - 1) ptx::umma_commit(ptx::smem_u32(&sh->acc_full[acc]));
@@ -382,7 +388,10 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
             if (!__all_sync(0xffffffffu, wait_bounded(ptx::smem_u32(&sh->pair_empty[slot]), phase, ctx,
                                                       kWaitPairEmpty)))
                 break;
-            if (lane == 0) sh->pairs_consumed = k + 1;
+            if (lane == 0) {
+                sh->pairs_consumed = k + 1;
+                ptx::mbar_arrive(ptx::smem_u32(&sh->tick));
+            }
             if (++slot == a.nbp) { slot = 0; phase ^= 1u; }
         }
     } else if (warp >= TC_FIRST_READER && warp < TC_FIRST_READER + TC_READERS) {
@@ -410,7 +419,8 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
                 // the buffers of the pairs this task writes are free once the pairs that used
                 // them before (nbp pairs earlier) have been consumed
                 if (sh->pairs_consumed < ((bfirst + cnt - 1) >> 1) - a.nbp + 1)
-                    ok = wait_counter(&sh->pairs_consumed, ((bfirst + cnt - 1) >> 1) - a.nbp + 1, ctx, kWaitPairEmpty);
+                    ok = wait_counter(&sh->pairs_consumed, ptx::smem_u32(&sh->tick), ((bfirst + cnt - 1) >> 1) - a.nbp + 1, ctx,
+                                      kWaitPairEmpty);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 const uint32_t strip = strips_u32 + (uint32_t)(sidx * a.strip_bytes);
@@ -423,11 +433,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
                     const int col0 = tw * M - 1;
                     int e0;
                     if (MODE == 0) e0 = pa * a.RS + col0 - (((it.tw0 * M - 1 + 8) & ~7) - 8);
-                    else if (MODE == 1) {
-                        const int j = pa / a.rpb;
-                        e0 = j * TC_CB * a.box_elems + (pa - j * a.rpb) * a.RS + col0 +
-                             (a.nbox == 1 ? (((it.th * M - 1) * g.W) & 7) : 0);
-                    }
+                    else if (MODE == 1) e0 = pa * a.RS + col0 + (((it.th * M - 1) * g.W) & 7);
                     else e0 = (th * M - 1 + pa) * a.RS + col0;
                     uint32_t mk[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, NN == 8 ? 0xffffffffu : 0u};
                     bool masked = false;
@@ -444,6 +450,8 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
                             }
                         }
                     }
+                    // the element offset may be negative (left / top padding): the words read
+                    // there are masked, and the strips are not at the start of shared memory
                     uint32_t src = strip + (uint32_t)(2 * (e0 + cq * 16 * a.CS));
                     const uint32_t src_step = (uint32_t)(2 * a.CS);
                     const uint32_t dst0 = bring_u32 + (uint32_t)(((bfirst + tsub) % (2 * a.nbp)) * TC_TILE_BYTES) +
@@ -493,7 +501,8 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
         // the other slot: fill the missing tile with zeros.  (The pair's buffer is free: its
         // first tile was written after a wait for pair_empty.)
         if (ok && (nbt & 1) && rw < TC_CQ)
-            ok = __all_sync(0xffffffffu, wait_counter(&sh->pairs_consumed, (nbt >> 1) - a.nbp + 1, ctx, kWaitPairEmpty));
+            ok = __all_sync(0xffffffffu, wait_counter(&sh->pairs_consumed, ptx::smem_u32(&sh->tick), (nbt >> 1) - a.nbp + 1,
+                                                      ctx, kWaitPairEmpty));
         if (ok && (nbt & 1) && rw < TC_CQ) {
             const uint32_t dst = bring_u32 + (uint32_t)((nbt % (2 * a.nbp)) * TC_TILE_BYTES) + (uint32_t)(rw * 16 * 128);
 #pragma unroll
@@ -511,11 +520,33 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
         const int L = quarter * 32 + lane;                 // TMEM lane = accumulator row
         const int slot = L / PL, p = L - slot * PL;
         const bool lane_ok = slot < S && p < P;
-        const float sp = tab.in_scale[lane_ok ? p : 0];
+        const float sp = tab.in_scale[lane_ok ? p : 0], sl = tab.in_scale_lo[lane_ok ? p : 0];
         const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(u * 64);
         const int ngroups = (nbt + 2 * S - 1) / (2 * S);
+        if (qw < 4) {
+            // The constant matrix goes to tensor memory once per CTA, one copy per slot: row
+            // p of the matrix on lane s * PL + p, zeros on every other lane.
+#pragma unroll 1
+            for (int sl = 0; sl < S; ++sl) {
+                const int pp = L - sl * PL;
+                const bool has = pp >= 0 && pp < P;
+                const uint32_t *row = a.amat + (size_t)(has ? pp : 0) * C::KW;
+#pragma unroll
+                for (int kc = 0; kc < C::KW / 8; ++kc) {
+                    uint32_t v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) v[i] = has ? __ldg(row + kc * 8 + i) : 0u;
+                    ptx::tmem_st_x8(tmem_base + ((uint32_t)(quarter * 32) << 16) +
+                                    (uint32_t)(TC_AMAT_COL + sl * C::KW + kc * 8), v);
+                }
+            }
+            ptx::tmem_st_wait();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->amat_full));
+        }
         for (int grp = team; grp < ngroups; grp += TC_TEAMS) {
-            const int acc = grp % TC_NACC;
+            const int acc = team;                          // TC_NACC == TC_TEAMS
             if (!wait_bounded(ptx::smem_u32(&sh->acc_full[acc]), (uint32_t)((grp / TC_NACC) & 1), ctx, kWaitAccFull))
                 break;
             ptx::tc_fence_after();
@@ -538,9 +569,9 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
                         if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[acc]));
                     }
                     float scale, inv;
-                    group_scale_inv(scale_and_max32(r, sp, 0.f), scale, inv);
+                    group_scale_inv(fabsf(scaled(absmax32(r, 0.f), sp, sl)), scale, inv);
                     if (valid) {
-                        codes32(r, inv, dst + 32 * h);
+                        codes32(r, sp, sl, inv, dst + 32 * h);
                         sd[(size_t)h * g.Ts] = scale;
                     }
                 }
@@ -549,13 +580,13 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
                 // then the first half again from TMEM
                 ptx::tmem_ld_x32(taddr, r);
                 ptx::tmem_ld_wait();
-                const float m = scale_and_max32(r, sp, 0.f);
+                const float m = absmax32(r, 0.f);
                 ptx::tmem_ld_x32(taddr + 32u, r);
                 ptx::tmem_ld_wait();
                 float scale, inv;
-                group_scale_inv(scale_and_max32(r, sp, m), scale, inv);
+                group_scale_inv(fabsf(scaled(absmax32(r, m), sp, sl)), scale, inv);
                 if (valid) {
-                    codes32(r, inv, dst + 32);
+                    codes32(r, sp, sl, inv, dst + 32);
                     a.sX[((size_t)p * g.G + cb) * g.Ts + t] = scale;
                 }
                 ptx::tmem_ld_x32(taddr, r);
@@ -563,8 +594,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[acc]));
-                scale_and_max32(r, sp, 0.f);
-                if (valid) codes32(r, inv, dst);
+                if (valid) codes32(r, sp, sl, inv, dst);
             }
         }
     }
@@ -573,7 +603,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, 128 * TC_NACC);
+        ptx::tmem_dealloc(tmem_base, TC_TMEM_COLS);
     }
 }
 
@@ -594,8 +624,7 @@ cudaError_t launch_tc(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
     a.mode = k.mode; a.TBW = k.TBW; a.NCHUNK = k.NCHUNK; a.NCB = k.NCB; a.items = k.items;
     a.CS = k.CS; a.RS = k.RS;
     a.strip_bytes = k.strip_bytes; a.nstrip = k.nstrip; a.nbp = k.nbp;
-    a.nbox = k.nbox; a.rpb = k.rpb; a.box_elems = k.box_elems;
-    a.amat = g_amat[plan.device][M == 6 ? 1 : 0];
+    a.amat = static_cast<const uint32_t *>(g_amat[plan.device][M == 6 ? 1 : 0]);
     a.debug_skip_item = plan.debug_skip_item;
     if (!a.amat) return cudaErrorInvalidValue;
     auto kern = input_transform_tc_kernel<M, GS, MODE>;
@@ -628,25 +657,22 @@ const float kBT6[64] = {
     0, -0.5f, 0.25f, 2.5f, -1.25f, -2, 1, 0, 0, 2, 4, -2.5f, -5, 0.5f, 1, 0,
     0, -2, 4, 2.5f, -5, -0.5f, 1, 0,         0, -1, 0, 5.25f, 0, -5.25f, 0, 1};
 
-// [AROWS][128 bytes]: row (S-1)*PL + p holds BT[i][a] * BT[j][b] for p = i*n + j at K index
-// a*8 + b (fp16; every product is exact), the 16-byte chunk a of a row stored at chunk
-// a ^ (row & 7) (the 128-byte swizzle of the MMA's K-major operand layout); all other
-// rows and entries are zero.
+// [P][KW] 32-bit words: word (p, a * 4 + b / 2) holds BT[i][a] * BT[j][b] for p = i*n + j and
+// two consecutive b (fp16; every product is exact; b >= n gives zero), i.e. K index a*8 + b.
 template <int M>
 void build_amat(std::vector<uint16_t> &out)
 {
     using C = TcCfg<M>;
     const float *bt = M == 6 ? kBT6 : kBT4;
-    out.assign((size_t)C::AROWS * 64, 0);
+    out.assign((size_t)C::P * C::KW * 2, 0);
     for (int p = 0; p < C::P; ++p) {
-        const int row = (C::S - 1) * C::PL + p;
         const int i = p / C::NN, j = p % C::NN;
         for (int a = 0; a < C::NN; ++a)
             for (int b = 0; b < C::NN; ++b) {
                 const __half h = __float2half_rn(bt[i * C::NN + a] * bt[j * C::NN + b]);
                 uint16_t bits;
                 memcpy(&bits, &h, 2);
-                out[(size_t)row * 64 + ((a ^ (row & 7)) * 8) + b] = bits;
+                out[(size_t)p * C::KW * 2 + a * 8 + b] = bits;
             }
     }
 }
@@ -663,43 +689,43 @@ void plan_input_transform_tc(wfq_plan &plan)
     if (plan.sm_count <= 0) return;
     const int n = g.n, m = g.m;
     const long long hw = (long long)g.H * g.W;
-    const int a_bytes = m == 6 ? TcCfg<6>::A_BYTES : TcCfg<4>::A_BYTES;
     k.nbp = 4;   // operand-tile ring: pairs in flight
     // shared memory left for the strip ring
-    const int budget = 227 * 1024 - 1024 /*alignment*/ - (int)sizeof(TcShared) - a_bytes - k.nbp * 2 * TC_TILE_BYTES;
+    const int budget = 227 * 1024 - 1024 /*alignment*/ - (int)sizeof(TcShared) - k.nbp * 2 * TC_TILE_BYTES;
     const int strip_max = budget / 2;       // at least two strips
-    k.nbox = 1; k.rpb = n; k.box_elems = 0; k.NCHUNK = 1;
+    k.NCHUNK = 1;
     int mode = -1;
-    // mode 1 with several boxes: rows are 16-byte multiples, a box takes rpb whole rows
-    int rpb = 0;
-    if (g.W % 8 == 0)
-        for (int r = n; r >= 1; --r)
-            if (n % r == 0 && r * g.W <= 256) { rpb = r; break; }
-    if (rpb > 0 && TC_CB * n * g.W * 2 <= strip_max) {
+    if (g.W % 8 == 0) {
+        // Column chunks of TBW tiles.  A chunk's first column, tw0 * m - 1, lies up to 7 past
+        // the 16-byte boundary the box starts at; the box width is 8 modulo 16 elements (bank
+        // spread of the patch rows).  Among the chunk sizes whose strip fits twice, take the
+        // one with the least work on the busiest CTA (a strip costs about three tiles).
+        long long best = -1;
+        for (int nch = 1; nch <= g.TW; ++nch) {
+            const int tbw = (g.TW + nch - 1) / nch;
+            if ((g.TW + tbw - 1) / tbw != nch) continue;
+            int bw = (tbw * m + 2 + 7 + 7) / 8 * 8;
+            if (bw % 16 == 0) bw += 8;
+            if (bw > 256 || TC_CB * n * bw * 2 > strip_max) continue;
+            const long long items = (long long)g.N * g.TH * nch * (g.C / TC_CB);
+            const long long cost = ((items + plan.sm_count - 1) / plan.sm_count) * (tbw + 3);
+            if (best < 0 || cost < best) {
+                best = cost;
+                mode = 0;
+                k.TBW = tbw; k.NCHUNK = nch;
+                k.CS = n * bw; k.RS = bw;
+                k.strip_bytes = TC_CB * n * bw * 2;
+                k.box[0] = (unsigned)bw; k.box[1] = (unsigned)n; k.box[2] = TC_CB;
+            }
+        }
+    } else if ((hw * 2) % 16 == 0 && n * g.W + 8 <= 256) {
+        // one box per strip; it starts at the 16-byte boundary below its first element
         mode = 1;
-        k.TBW = g.TW; k.nbox = n / rpb; k.rpb = rpb; k.box_elems = rpb * g.W;
-        k.CS = k.box_elems; k.RS = g.W;
-        k.strip_bytes = k.nbox * TC_CB * k.box_elems * 2;
-        k.box[0] = (unsigned)k.box_elems; k.box[1] = TC_CB; k.box[2] = 1;
-    } else if ((hw * 2) % 16 == 0 && g.W % 8 != 0 && n * g.W + 8 <= 256) {
-        // one box; the strip starts at the 16-byte boundary below its first element
-        mode = 1;
-        k.TBW = g.TW; k.box_elems = (n * g.W + 7 + 7) / 8 * 8;
-        k.CS = k.box_elems; k.RS = g.W;
-        k.strip_bytes = TC_CB * k.box_elems * 2;
-        k.box[0] = (unsigned)k.box_elems; k.box[1] = TC_CB; k.box[2] = 1;
-    } else if (g.W % 8 == 0) {
-        // column chunks: as many tiles (a multiple of 4) as half the strip budget holds
-        mode = 0;
-        int tbw = 4;
-        while (tbw + 4 <= g.TW + 3 && TC_CB * n * (((tbw + 4) * m + 2 + 14) / 8 * 8) * 2 <= strip_max) tbw += 4;
-        const int nch = (g.TW + tbw - 1) / tbw;
-        tbw = ((g.TW + nch - 1) / nch + 3) / 4 * 4;      // even chunks
-        k.TBW = tbw; k.NCHUNK = (g.TW + tbw - 1) / tbw;
-        const int BW = (tbw * m + 2 + 14) / 8 * 8;
-        k.CS = n * BW; k.RS = BW;
-        k.strip_bytes = TC_CB * n * BW * 2;
-        k.box[0] = (unsigned)BW; k.box[1] = (unsigned)n; k.box[2] = TC_CB;
+        const int bw = (n * g.W + 7 + 7) / 8 * 8;
+        k.TBW = g.TW;
+        k.CS = bw; k.RS = g.W;
+        k.strip_bytes = TC_CB * bw * 2;
+        k.box[0] = (unsigned)bw; k.box[1] = TC_CB; k.box[2] = 1;
     } else if ((hw * TC_CB * 2) % 128 == 0 && hw * TC_CB * 2 <= strip_max) {
         mode = 2;
         k.TBW = g.TH * g.TW;
@@ -712,7 +738,7 @@ void plan_input_transform_tc(wfq_plan &plan)
     int nstrip = budget / k.strip_bytes;
     if (nstrip > TC_MAX_STRIP) nstrip = TC_MAX_STRIP;
     k.nstrip = nstrip;
-    k.smem = 1024 + a_bytes + k.nbp * 2 * TC_TILE_BYTES + nstrip * k.strip_bytes + (int)sizeof(TcShared);
+    k.smem = 1024 + k.nbp * 2 * TC_TILE_BYTES + nstrip * k.strip_bytes + (int)sizeof(TcShared);
     k.grid = k.items < plan.sm_count ? k.items : plan.sm_count;
     k.use = true;
 }

@@ -43,6 +43,11 @@ struct Geometry {
 struct ScaleTables {
     float in_scale[kMaxP];   // (sB_i/sBstd_i)*(sB_j/sBstd_j): applied after the
                              // standard-scaled integer/rational input transform
+    float in_scale_lo[kMaxP];  // the part of that factor that in_scale lost to rounding: the
+                             // kernels form X = fma(Z, in_scale, Z * in_scale_lo), which is the
+                             // correctly rounded product with the unrounded factor in all but
+                             // rare double-rounding cases (the quantizer's codes are sensitive
+                             // to the last bit of X where a group holds an outlier)
     float out_scale[kMaxP];  // sA_i*sA_j: applied before the output transform
 };
 
@@ -69,7 +74,6 @@ struct K1TcPlan {
     int TBW = 0, NCHUNK = 0, NCB = 0, items = 0;
     int CS = 0, RS = 0;      // strip strides in elements: channel, patch row
     int strip_bytes = 0, nstrip = 0, nbp = 0;
-    int nbox = 1, rpb = 0, box_elems = 0;   // mode 1: boxes per strip, rows per box, elements per box row
     int smem = 0, grid = 0;
     unsigned box[3] = {0, 0, 0};
 };
@@ -110,7 +114,7 @@ struct wfq_plan {
     long long wait_cycles = 2000000000LL;   // limit of every device-side wait (~1 s)
     int debug_skip_item = -1;  // >= 0: the input transform's producer skips this work item
     int debug_skip_gemm_stage = -1;   // >= 0: the contraction's producer (CTA 0) skips this stage
-    int debug_force_generic_k1 = 0;   // 1: always use the cp.async input-transform kernel
+    int k1_choice = 0;         // input-transform kernel: 0 automatic, 1 cp.async, 2 tensor cores where they apply
 
     CUtensorMap tmap_xq;       // Xq as (C, T, P) bytes, 128B-swizzled boxes
     CUtensorMap tmap_wq;       // Wq as (C, K, P)

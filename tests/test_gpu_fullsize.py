@@ -17,11 +17,21 @@ pytestmark = pytest.mark.gpu
 FULL = [L for cfg in (2, 3, 4, 5) for L in wl.config_layers(cfg)]
 
 
+# the tensor-core input transform at full size: one layer per staging mode and tile size
+TC_FULL = [wl.config_layers(2)[i] for i in (0, 1, 2, 3)] + wl.config_layers(4) + [wl.config_layers(5)[i] for i in (5, 6)]
+
+
+@pytest.mark.parametrize("layer", TC_FULL, ids=lambda L: L.name)
+def test_full_size_sampled_tiles_tensor_core_input_transform(layer):
+    test_full_size_sampled_tiles(layer, k1_kernel=2)
+
+
 @pytest.mark.parametrize("layer", FULL, ids=lambda L: L.name)
-def test_full_size_sampled_tiles(layer):
+def test_full_size_sampled_tiles(layer, k1_kernel=0):
     import torch
     from tests.gpu_util import make_conv, codes_close, scales_close, max_rel, FINAL_TOL
     conv, (x, w, sB, sG) = make_conv(layer)
+    b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, k1_kernel)
     xd = torch.from_numpy(x).cuda()
     y = conv.forward(xd)
     torch.cuda.synchronize()
@@ -43,15 +53,7 @@ def test_full_size_sampled_tiles(layer):
     Wq = conv.buffer(b.WFQ_BUF_WQ)[:, torch.from_numpy(ks).cuda()].cpu().numpy()
     codes_close(Wq, ref.Wq)
 
-    m = layer.m
-    geo = orc.geometry(layer.N, layer.H, layer.W, m)
-    scale = np.max(np.abs(yh))
-    worst = 0.0
-    for i, t in enumerate(tiles):
-        tw, th, img = t % geo.TW, (t // geo.TW) % geo.TH, t // (geo.TW * geo.TH)
-        hh, ww = min(m, layer.H - th * m), min(m, layer.W - tw * m)
-        got = yh[img][ks][:, th * m:th * m + hh, tw * m:tw * m + ww]
-        want = ref.ytile[i][:, :hh, :ww]
-        worst = max(worst, float(np.max(np.abs(got - want))) / scale)
-    assert worst <= FINAL_TOL, worst
+    from tests.gpu_util import sampled_tiles_final_check
+    worst, continued = sampled_tiles_final_check(layer, conv, yh, ref, tiles, ks)
+    print(layer.name, f"worst {worst:.2e}", "tiles compared from the GPU's codes:", continued)
     conv.close()

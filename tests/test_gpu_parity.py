@@ -67,6 +67,13 @@ def test_reduced_configs(layer):
     _check(layer)
 
 
+@pytest.mark.parametrize("layer", [L for L in SMALL if L.dtype == "f16" and L.gs in (32, 64) and L.C % 64 == 0],
+                         ids=lambda L: L.name)
+def test_reduced_configs_tensor_core_input_transform(layer):
+    """The same layers with the tensor-core input transform selected."""
+    _check(layer, k1_kernel=2)
+
+
 def test_tiny_brute_force_shape():
     """C = K = group = 32, one tile per image."""
     for m in (4, 6):
@@ -141,10 +148,10 @@ def test_input_transform_kernels_agree():
     ref = orc.wfq(x, w[:1], L.m, L.gs, sB=sB, sG=sG)
     xbuf = torch.zeros(x.size + 8, dtype=torch.float16, device="cuda")
     got = []
-    for force, offset in ((0, 0), (1, 0), (0, 2)):          # offset in elements: 4-byte aligned only
+    for force, offset in ((2, 0), (1, 0), (2, 2)):          # offset in elements: 4-byte aligned only
         xd = xbuf[offset:offset + x.size].view(x.shape)
         xd.copy_(torch.from_numpy(x))
-        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_GENERIC_INPUT_TRANSFORM, force)
+        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, force)
         conv.buffer(b.WFQ_BUF_XQ).fill_(99)
         b.wfq_input_transform_quantize(conv.plan, xd.data_ptr(), conv._stream())
         torch.cuda.synchronize()
@@ -168,8 +175,10 @@ def test_bounded_waits_run_out_and_report():
     from oracle import oracle as orc
     L = Layer(1, 64, 64, 16, 16, 4, 64, "f16", "silu_outlier", "kaiming_chan", 9, 5, 0)
     # (option, value, stage call, expected wait ids)
-    cases = [(b.WFQ_DEBUG_SKIP_INPUT_ITEM, 1, "k1", {9}),    # im2col warps wait for the strip
-             (b.WFQ_DEBUG_SKIP_GEMM_STAGE, 0, "k2", {2})]    # MMA issuer waits for operands
+    # (the roles downstream of the starved one run out at about the same time: any of them
+    # may be the first to record its wait)
+    cases = [(b.WFQ_DEBUG_SKIP_INPUT_ITEM, 1, "k1", {9, 11, 13}),   # strip / operand pair / accumulator
+             (b.WFQ_DEBUG_SKIP_GEMM_STAGE, 0, "k2", {2, 4, 7})]     # operands / accumulator / scales
     for option, value, stage, want in cases:
         conv, (x, w, sB, sG) = make_conv(L)
         xd = torch.from_numpy(x).cuda()
@@ -177,6 +186,7 @@ def test_bounded_waits_run_out_and_report():
         torch.cuda.synchronize()
         conv.check_status()
         b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_WAIT_CYCLES, 2_000_000)   # about 1 ms
+        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, 2)
         b.wfq_plan_set_debug_option(conv.plan, option, value)
         if stage == "k1":
             b.wfq_input_transform_quantize(conv.plan, xd.data_ptr(), conv._stream())
