@@ -65,6 +65,9 @@ def parse_args():
                     help="skip the tensor-pipe rate, stand-alone contraction, sustained and parity legs")
     ap.add_argument("--no-graph", action="store_true",
                     help="enqueue every step with stream launches instead of replaying a CUDA graph")
+    ap.add_argument("--k1-kernel", type=int, default=0, choices=[0, 1, 2],
+                    help="input-transform kernel: 0 the library's choice, 1 cp.async, 2 tensor cores "
+                         "where they apply (profiling)")
     ap.add_argument("--cpu-seconds", type=float, default=16.0,
                     help="CPU time budget of the oracle baseline")
     return ap.parse_args()
@@ -270,7 +273,7 @@ def select_layers(wl, cfg, only_layer=None):
 class Workload:
     """The layers of one configuration: plans, device tensors, and the step as a CUDA graph."""
 
-    def __init__(self, cfg, only_layer, dev, stream, flush, use_graph=True):
+    def __init__(self, cfg, only_layer, dev, stream, flush, use_graph=True, k1_kernel=0):
         import torch
         from paper_2412_19867_b200 import binding as b
         from paper_2412_19867_b200 import workloads as wl
@@ -282,6 +285,8 @@ class Workload:
         for L, (x, w, sB, sG) in zip(self.layers, self.tensors):
             conv = b.Conv(L.N, L.C, L.K, L.H, L.W, L.m, L.gs, L.dtype, dev)
             conv.prepare(torch.from_numpy(w).to(dev), list(sB), list(sG))
+            if k1_kernel:
+                b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, k1_kernel)
             self.convs.append(conv)
             self.xs.append(torch.from_numpy(x).to(dev))
             self.ys.append(torch.empty((L.N, L.K, L.H, L.W), dtype=torch.float32, device=dev))
@@ -474,7 +479,8 @@ def run_wfq(args):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    wk = Workload(args.config, args.only_layer, dev, stream, flush, use_graph=not args.no_graph)
+    wk = Workload(args.config, args.only_layer, dev, stream, flush, use_graph=not args.no_graph,
+                  k1_kernel=args.k1_kernel)
     for _ in range(warmup):
         flush.zero_()
         wk.step()

@@ -83,6 +83,7 @@ struct GemmArgs {
     int *status;
     long long wait_cycles;    // limit of every mbarrier wait (about a second by default)
     int debug_skip_stage;     // >= 0: CTA 0's producer skips the loads of this stage (test hook)
+    long long l2_prefetch_bytes;   // per CTA: filter bytes it may ask into L2 ahead of the previous kernel's end
 };
 
 // MMA issue loop for the common shapes in which the chunks tile a stage exactly
@@ -198,7 +199,37 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     ptx::tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
 
-    // everything above may overlap the tail of the kernel that produces Xq and sX
+    // Everything above may overlap the kernel that produces Xq and sX.  So may the filter
+    // stream, which does not depend on it: before waiting for that kernel the producer loads
+    // the filter half of its first stages and asks for the filter tiles of its first units
+    // to be brought into L2 (bounded by a per-CTA share of `l2_prefetch_bytes`).
+    constexpr int W_ROWS = SWAP ? BM : BN;                 // filter rows of a stage
+    // stages of the first unit whose filter half is loaded early
+    const int pre = (a.l2_prefetch_bytes > 0 && (int)blockIdx.x < units) ? (KB < NSTAGES ? KB : NSTAGES) : 0;
+    if (warp == 0 && lane == 0) {
+        ptx::prefetch_tmap(&tmA);
+        ptx::prefetch_tmap(&tmB);
+        const CUtensorMap *tmW = SWAP ? &tmA : &tmB;
+        long long budget = a.l2_prefetch_bytes;
+        for (int u = blockIdx.x, first = 1; u < units && budget > 0; u += gridDim.x, first = 0) {
+            const int nt = u % NT, mt = (u / NT) % MT, p = u / (NT * MT);
+            const int wrow = SWAP ? mt * BM : nt * BN;
+            for (int kb = 0; kb < KB && budget > 0; ++kb) {
+                if (first && kb < pre) {
+                    if (!(blockIdx.x == 0 && kb == a.debug_skip_stage)) {
+                        const uint32_t bar = ptx::smem_u32(&sh->full[kb]);
+                        const uint32_t dst = ptx::smem_u32(tiles + (size_t)kb * C::STAGE_BYTES) + (SWAP ? 0 : A_BYTES);
+                        ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+                        ptx::tma_load_3d(dst, tmW, bar, kb * BK, wrow, p);
+                    }
+                } else {
+                    ptx::tma_prefetch_l2_3d(tmW, kb * BK, wrow, p);
+                    budget -= W_ROWS * BK;
+                }
+            }
+        }
+    }
+    if (warp == 0) __syncwarp();
     ptx::grid_dependency_wait();
 
     if (warp == 0) {
@@ -206,10 +237,6 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // All 32 lanes walk the loop and wait together; lane 0 alone issues the copies.
         // (A warp whose other lanes sit at the final block barrier while one lane works
         // gets scheduled far too rarely.)
-        if (lane == 0) {
-            ptx::prefetch_tmap(&tmA);
-            ptx::prefetch_tmap(&tmB);
-        }
         int stage = 0;
         uint32_t phase = 0;
         long long issued = 0;
@@ -223,9 +250,15 @@ gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (lane == 0 && !(blockIdx.x == 0 && issued == a.debug_skip_stage)) {
                     const uint32_t bar = ptx::smem_u32(&sh->full[stage]);
                     const uint32_t a_dst = ptx::smem_u32(tiles + (size_t)stage * C::STAGE_BYTES);
-                    ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
-                    ptx::tma_load_3d(a_dst, &tmA, bar, kb * BK, mt * BM, p);
-                    ptx::tma_load_3d(a_dst + A_BYTES, &tmB, bar, kb * BK, nt * BN, p);
+                    if (issued >= pre) {
+                        ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+                        ptx::tma_load_3d(a_dst, &tmA, bar, kb * BK, mt * BM, p);
+                        ptx::tma_load_3d(a_dst + A_BYTES, &tmB, bar, kb * BK, nt * BN, p);
+                    } else if (SWAP) {      // the filter half of this stage is already on its way
+                        ptx::tma_load_3d(a_dst + A_BYTES, &tmB, bar, kb * BK, nt * BN, p);
+                    } else {
+                        ptx::tma_load_3d(a_dst, &tmA, bar, kb * BK, mt * BM, p);
+                    }
                 }
                 __syncwarp();
                 ++issued;
@@ -493,6 +526,8 @@ cudaError_t launch_variant(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t
     const int units = g.P * MT * NT;
     const int slots = 2 * plan.sm_count;          // two CTAs per SM
     const int grid = units < slots ? units : slots;
+    // the filters share L2 (126 MB) with Xq, sX and Y: at most 48 MB of them are asked for early
+    a.l2_prefetch_bytes = pdl ? (48LL << 20) / grid : 0;
     auto kern = gemm_dequant_kernel<BN, SWAP, DUMP>;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);

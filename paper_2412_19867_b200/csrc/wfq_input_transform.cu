@@ -313,6 +313,9 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
     constexpr int NN = M + 2;
     constexpr int P = NN * NN;
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    // The contraction kernel launched behind this one may start its prologue and its filter
+    // stream now (it waits for this grid's completion before it touches Xq or sX).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // two strip buffers (the next item is staged while this one is transformed), then Z
     float *Zs = reinterpret_cast<float *>(smem_raw + (1 + prm.dbuf) * prm.strip_bytes);   // [tile][position][CBP]
     const int CBP = prm.CB + 4;   // 16-byte aligned rows an odd number of 16-byte units apart

@@ -256,6 +256,7 @@ input_transform_tc_kernel(const __grid_constant__ CUtensorMap tmx, TcArgs a, Geo
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const WaitCtx ctx{&sh->abort, a.status, a.wait_cycles};
+    ptx::grid_launch_dependents();   // the next kernel's prologue and filter stream may start
 
     // One strip load (all lanes call it; lane 0 issues).
     auto issue_strip = [&](int item, int sidx) {
