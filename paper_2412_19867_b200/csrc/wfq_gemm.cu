@@ -624,6 +624,8 @@ cudaError_t setup_gemm()
 {
     cudaError_t e = setup_variant<32, true, true>();
     if (e == cudaSuccess) e = setup_variant<32, true, false>();
+    if (e == cudaSuccess) e = setup_variant<48, true, true>();
+    if (e == cudaSuccess) e = setup_variant<48, true, false>();
     if (e == cudaSuccess) e = setup_variant<64, true, true>();
     if (e == cudaSuccess) e = setup_variant<64, true, false>();
     if (e == cudaSuccess) e = setup_variant<64, false, true>();
@@ -650,7 +652,11 @@ void gemm_choose(const Geometry &g, bool *swap, int *bn)
 {
     auto up = [](long long v, int b) { return (v + b - 1) / b * b; };
     const long long normal = up(g.T, BM) * up(g.K, 64);
-    const int bn_sw = g.T <= 32 ? 32 : 64;
+    // swapped: the tile columns are padded to a multiple of the column block (32, 48 or 64:
+    // every padded column is promoted like a real one); the largest block among the least padded
+    int bn_sw = 64;
+    for (int c : {48, 32})
+        if (up(g.T, c) < up(g.T, bn_sw)) bn_sw = c;
     const long long swapped = up(g.K, BM) * up(g.T, bn_sw);
     *swap = 5 * swapped < 4 * normal;   // swapped stores are less efficient: want >= 20 % less work
     *bn = *swap ? bn_sw : 64;
@@ -663,6 +669,9 @@ cudaError_t launch_gemm(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t st
         if (plan.gemm_bn == 32)
             return dump ? launch_variant<32, true, true>(plan, acc_dump, stream, pdl)
                         : launch_variant<32, true, false>(plan, acc_dump, stream, pdl);
+        if (plan.gemm_bn == 48)
+            return dump ? launch_variant<48, true, true>(plan, acc_dump, stream, pdl)
+                        : launch_variant<48, true, false>(plan, acc_dump, stream, pdl);
         return dump ? launch_variant<64, true, true>(plan, acc_dump, stream, pdl)
                     : launch_variant<64, true, false>(plan, acc_dump, stream, pdl);
     }

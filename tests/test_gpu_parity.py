@@ -54,6 +54,10 @@ SMALL = [
     Layer(1, 192, 40, 13, 13, 6, 96, "f16", "silu_outlier", "kaiming_chan", 4, 0, 7),
     Layer(1, 320, 64, 8, 8, 4, 160, "f16", "silu_outlier", "kaiming_chan", 4, 0, 8),    # swapped
     Layer(2, 512, 64, 12, 12, 4, 256, "f16", "silu_outlier", "kaiming_chan", 4, 0, 9),
+    # swapped contraction with the 48-column block: one and two column blocks, groups of 64 and 32
+    Layer(1, 128, 256, 24, 24, 4, 64, "f16", "silu_outlier", "kaiming_chan", 5, 8, 3),  # T = 36
+    Layer(1, 128, 256, 24, 24, 4, 32, "f16", "silu_outlier", "kaiming_chan", 5, 8, 4),
+    Layer(1, 64, 128, 36, 40, 4, 64, "f16", "silu_outlier", "kaiming_chan", 5, 8, 5),   # T = 90
     # tensor-core input transform: column chunks with a ragged last chunk (3-D boxes), whole
     # tile rows in several boxes, an odd number of operand tiles per CTA, groups of 32
     Layer(1, 64, 32, 24, 136, 4, 64, "f16", "silu_outlier", "kaiming_chan", 5, 0, 1),   # W = 136: chunks
