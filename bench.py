@@ -45,6 +45,12 @@ FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
 NOMINAL_INT8_TOPS = 4500.0
 KERNELS = ["input_transform_quantize", "gemm_dequantize", "output_transform"]
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, mean over the launches of one step,
+# from one ncu capture of this command (profiles/gemm_dequant_cfg5_dram_traffic.txt).  Keyed by
+# (configuration, kernel); anything else has no capture of the current kernels and reports null.
+# The written Y stays in the 126 MB L2 for the output transform, so this is below the
+# algorithmic bytes.
+NCU_TRAFFIC = {(5, "gemm_dequantize"): 39228851}
 
 
 def parse_args():
@@ -531,12 +537,13 @@ def run_wfq(args):
     achieved = tot_bytes[dom] / (tot_ms[dom] * 1e-3) / 1e9
     nl = len(wk.layers)
     roofline = {"bound": "hbm", "kernel": KERNELS[dom], "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC.get((args.config, KERNELS[dom])) if args.only_layer is None else None,
+                "peak_source": peak_src,
                 "launches_per_step": nl, "algorithmic_bytes_per_step": tot_bytes[dom],
                 "algorithmic_bytes_per_launch": tot_bytes[dom] / nl,
                 "us_per_launch": tot_ms[dom] * 1e3 / nl,
-                "note": "traffic: no ncu capture of this kernel version on the headline workload; "
-                        "per-launch DRAM bytes of single layers are in profiles/",
+                "note": "traffic: mean DRAM bytes per launch over the launches of one step (ncu, "
+                        "profiles/); null where the current kernels have no capture on this workload",
                 "all_kernels": head["kernels"]}
 
     # ---- sustained: the same step replayed for about two seconds -------------------------

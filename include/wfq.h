@@ -63,6 +63,9 @@ typedef enum {
 
 typedef enum { WFQ_F32 = 0, WFQ_F16 = 1 } wfq_dtype_t;
 
+/* Activation applied by the output transform after the optional bias. */
+typedef enum { WFQ_ACT_NONE = 0, WFQ_ACT_RELU = 1, WFQ_ACT_SILU = 2 } wfq_activation_t;
+
 /* Buffers that wfq_debug_get can expose (all device memory). */
 typedef enum {
     WFQ_BUF_XQ = 0,     /* int8  Xq[P][T][C]            (workspace)  */
@@ -106,6 +109,16 @@ wfq_status_t wfq_plan_create(wfq_plan_t **out, int N, int C, int K, int H, int W
 
 /* Element type of x in wfq_conv_forward (default WFQ_F32).  Call before forward. */
 wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype);
+
+/*
+ * Optional epilogue fused into the output transform (the paper's layers are followed by a
+ * bias and an activation; the paper itself gives no formula for them, Section 3.1 defines
+ * the convolution only): y = act(conv(x, w) + bias[k]).
+ *   bias_dev  device, fp32 [K], caller-owned and kept alive while the plan is used; NULL = none
+ *   act       WFQ_ACT_NONE, WFQ_ACT_RELU (max(t, 0)) or WFQ_ACT_SILU (t / (1 + exp(-t)))
+ * Host only; takes effect from the next forward call.  Default: no bias, no activation.
+ */
+wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_activation_t act);
 
 /*
  * Bytes of caller-owned device scratch the plan needs (Xq + sX + Y, each region

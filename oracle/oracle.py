@@ -243,6 +243,20 @@ def unquantized(x, w, m, sB=None, sG=None, sA=None, derive_sA_exact=True):
     return scatter_tiles(output_transform(Y, m, mats), N, H, W, m)
 
 
+def epilogue(y, bias=None, act="none"):
+    """Bias per output channel and activation on y[N][K][H][W] (fp64): none, relu, silu."""
+    y = np.asarray(y, dtype=np.float64)
+    if bias is not None:
+        y = y + np.asarray(bias, dtype=np.float64)[None, :, None, None]
+    if act == "relu":
+        return np.maximum(y, 0.0)
+    if act == "silu":
+        return y / (1.0 + np.exp(-y))
+    if act != "none":
+        raise ValueError(act)
+    return y
+
+
 def sqnr_db(ref, test):
     ref = np.asarray(ref, dtype=np.float64)
     err = np.asarray(test, dtype=np.float64) - ref

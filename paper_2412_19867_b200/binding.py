@@ -15,6 +15,7 @@ WFQ_OK, WFQ_ERR_INVALID_ARG, WFQ_ERR_UNSUPPORTED, WFQ_ERR_ALLOC = 0, 1, 2, 3
 WFQ_ERR_NOT_PREPARED, WFQ_ERR_CUDA, WFQ_ERR_TIMEOUT, WFQ_ERR_SCRATCH_TOO_SMALL = 4, 5, 6, 7
 WFQ_STATIC_SCRATCH_FLOATS = 4 * 1024 * 1024
 WFQ_F32, WFQ_F16 = 0, 1
+WFQ_ACT_NONE, WFQ_ACT_RELU, WFQ_ACT_SILU = 0, 1, 2
 WFQ_BUF_XQ, WFQ_BUF_SX, WFQ_BUF_WQ, WFQ_BUF_SW, WFQ_BUF_Y, WFQ_BUF_STATUS = range(6)
 WFQ_DEBUG_WAIT_CYCLES, WFQ_DEBUG_SKIP_INPUT_ITEM, WFQ_DEBUG_INPUT_TRANSFORM_KERNEL = range(3)
 WFQ_DEBUG_SKIP_GEMM_STAGE = 3
@@ -27,6 +28,7 @@ EXPORTS = [
     "wfq_output_transform", "wfq_debug_gemm_acc32", "wfq_debug_get",
     "wfq_check_device_status", "wfq_plan_destroy", "wfq_status_string", "wfq_version",
     "wfq_quantize_filters_static", "wfq_plan_set_debug_option", "wfq_debug_int8_mma_rate",
+    "wfq_plan_set_epilogue",
 ]
 
 _lib = None
@@ -64,6 +66,7 @@ def load():
     lib.wfq_check_device_status.argtypes = [vp, vp, ctypes.POINTER(ci)]
     lib.wfq_plan_destroy.argtypes = [vp]
     lib.wfq_quantize_filters_static.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
+    lib.wfq_plan_set_epilogue.argtypes = [vp, vp, ci]
     lib.wfq_plan_set_debug_option.argtypes = [vp, ci, ctypes.c_longlong]
     lib.wfq_debug_int8_mma_rate.argtypes = [vp, ci, ci, ctypes.POINTER(ctypes.c_longlong), vp]
     lib.wfq_status_string.argtypes = [ci]
@@ -104,6 +107,10 @@ def wfq_plan_create(N, C, K, H, W, m, r=3, group_size=64, bits=8):
 
 def wfq_plan_set_input_dtype(plan, dtype):
     _check(load().wfq_plan_set_input_dtype(plan, dtype), "wfq_plan_set_input_dtype")
+
+
+def wfq_plan_set_epilogue(plan, bias_dev, act=WFQ_ACT_NONE):
+    _check(load().wfq_plan_set_epilogue(plan, bias_dev, act), "wfq_plan_set_epilogue")
 
 
 def wfq_plan_workspace_bytes(plan):
@@ -224,6 +231,14 @@ class Conv:
         assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
         with torch.cuda.device(self.device):
             wfq_prepare_filters(self.plan, w.data_ptr(), sB, sG, sA, self._stream())
+
+    def set_epilogue(self, bias=None, act=WFQ_ACT_NONE):
+        """bias: fp32 CUDA tensor [K] or None; kept alive by this object."""
+        if bias is not None:
+            assert bias.is_cuda and bias.dtype == self.torch.float32 and bias.is_contiguous()
+            assert bias.numel() == self.shape[2]
+        self._bias = bias
+        wfq_plan_set_epilogue(self.plan, None if bias is None else bias.data_ptr(), act)
 
     def forward(self, x, y=None):
         torch = self.torch

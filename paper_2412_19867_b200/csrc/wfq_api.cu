@@ -190,6 +190,18 @@ wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype)
     return WFQ_OK;
 }
 
+wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_activation_t act)
+{
+    if (!plan) return WFQ_ERR_INVALID_ARG;
+    if (act != WFQ_ACT_NONE && act != WFQ_ACT_RELU && act != WFQ_ACT_SILU) return WFQ_ERR_INVALID_ARG;
+    if (bias_dev && (reinterpret_cast<uintptr_t>(bias_dev) & 3u)) return WFQ_ERR_INVALID_ARG;
+    plan->bias = bias_dev;
+    plan->act = (int)act;
+    for (int i = 0; i < 2; ++i)
+        if (plan->sub[i]) { plan->sub[i]->bias = bias_dev; plan->sub[i]->act = (int)act; }
+    return WFQ_OK;
+}
+
 size_t wfq_plan_workspace_bytes(const wfq_plan_t *plan) { return plan ? plan->ws.total : 0; }
 
 wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t bytes)
@@ -372,6 +384,7 @@ static wfq_status_t setup_host_pipeline(wfq_plan *plan)
         q->tables = plan->tables;
         q->tmap_wq = plan->tmap_wq; q->tmap_wq_ok = plan->tmap_wq_ok;
         q->wait_cycles = plan->wait_cycles;
+        q->bias = plan->bias; q->act = plan->act;
         q->prepared = true;
         if (!plan->host_stream[s] &&
             cudaStreamCreateWithFlags(&plan->host_stream[s], cudaStreamNonBlocking) != cudaSuccess)

@@ -100,6 +100,8 @@ struct wfq_plan {
     int8_t *Wq = nullptr;      // [P][K][C]
     float *sW = nullptr;       // [P][G][Kp]
     int *status = nullptr;     // int32[4]
+    const float *bias = nullptr;   // caller-owned fp32[K] added in the output transform, or null
+    int act = 0;               // activation after the bias: 0 none, 1 ReLU, 2 SiLU
     void *x_stage = nullptr;   // staging for wfq_conv_forward_host
     float *y_stage = nullptr;
 

@@ -41,6 +41,20 @@ __device__ __forceinline__ void at_1d(const float (&v)[M + 2], float (&o)[M])
     if constexpr (M == 4) at_f43(v, o); else at_f63(v, o);
 }
 
+// Optional epilogue on the spatial-domain outputs of one row segment: per-output-channel
+// bias, then ReLU or SiLU (act: 0 none, 1 ReLU, 2 SiLU).
+template <int M>
+__device__ __forceinline__ void epilogue(float (&o)[M], float bias, int act)
+{
+#pragma unroll
+    for (int v = 0; v < M; ++v) {
+        float t = o[v] + bias;
+        if (act == 1) t = fmaxf(t, 0.f);
+        else if (act == 2) t = t * __frcp_rn(1.f + __expf(-t));   // exp overflow: t * 0
+        o[v] = t;
+    }
+}
+
 // STORE: 2 = 16-byte stores straight from the
 // registers (F(4,3), W a multiple of 4: neighbouring lanes then write neighbouring 16 bytes
 // and a warp fills whole sectors), 1 = every other even W, 0 = odd W: the m-float row
@@ -51,10 +65,10 @@ __device__ __forceinline__ void at_1d(const float (&v)[M + 2], float (&o)[M])
 // one array per output row u with the tiles side by side exactly as they lie in the image
 // row, and copies them out with consecutive lanes on consecutive 8 bytes (even W) or
 // consecutive floats (odd W).
-template <int M, int STORE>
-__global__ void __launch_bounds__(128, M == 6 ? 7 : 8)
+template <int M, int STORE, bool EPI>
+__global__ void __launch_bounds__(128, M == 6 ? (EPI ? 6 : 7) : 8)
 output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geometry g,
-                        ScaleTables tab)
+                        ScaleTables tab, const float *__restrict__ bias, int act)
 {
     constexpr int NN = M + 2;
     constexpr int TT = 128;                       // tiles per CTA
@@ -108,10 +122,12 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
     if constexpr (STORE != 2) {
         const int j = threadIdx.x;
         if (live) {
+            const float bk = (EPI && bias) ? __ldg(bias + k) : 0.f;
 #pragma unroll
             for (int u = 0; u < M; ++u) {
                 float o[M];
                 at_1d<M>(tmp[u], o);
+                if constexpr (EPI) epilogue<M>(o, bk, act);
                 float2 *dst = reinterpret_cast<float2 *>(out_s + (u * TT + j) * M);
 #pragma unroll
                 for (int v2 = 0; v2 < M; v2 += 2) dst[v2 / 2] = make_float2(o[v2], o[v2 + 1]);
@@ -153,10 +169,12 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
     } else {
         float *row = y + base;
         const bool full_w = (w0 + M <= g.W);
+        const float bk = (EPI && bias) ? __ldg(bias + k) : 0.f;
 #pragma unroll
         for (int u = 0; u < M; ++u) {
             float o[M];
             at_1d<M>(tmp[u], o);
+            if constexpr (EPI) epilogue<M>(o, bk, act);
             if (h0 + u < g.H) {
                 if (full_w) {
                     *reinterpret_cast<float4 *>(row) = make_float4(o[0], o[1], o[2], o[3]);
@@ -173,19 +191,40 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
 
 }  // namespace
 
+namespace {
+
+template <int M, int STORE, bool EPI>
+cudaError_t carveout()
+{
+    return cudaFuncSetAttribute(output_transform_kernel<M, STORE, EPI>,
+                                cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+}
+
+template <int M, int STORE>
+cudaError_t launch_variant(const cudaLaunchConfig_t &cfg, const wfq_plan &plan, float *y_dev)
+{
+    const float *Y = plan.ws.Y;
+    if (plan.bias || plan.act)
+        return cudaLaunchKernelEx(&cfg, output_transform_kernel<M, STORE, true>, Y, y_dev, plan.geo, plan.tables,
+                                  plan.bias, plan.act);
+    return cudaLaunchKernelEx(&cfg, output_transform_kernel<M, STORE, false>, Y, y_dev, plan.geo, plan.tables,
+                              plan.bias, plan.act);
+}
+
+}  // namespace
+
 // One-time attribute setting (per device): the staged variants want six or more CTAs of
 // 10-19 KB of shared memory per SM.
 cudaError_t setup_output_transform()
 {
-    const int carve = (int)cudaSharedmemCarveoutMaxShared;
-    cudaError_t e = cudaFuncSetAttribute(output_transform_kernel<4, 1>,
-                                         cudaFuncAttributePreferredSharedMemoryCarveout, carve);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(output_transform_kernel<6, 1>, cudaFuncAttributePreferredSharedMemoryCarveout, carve);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(output_transform_kernel<4, 0>, cudaFuncAttributePreferredSharedMemoryCarveout, carve);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(output_transform_kernel<6, 0>, cudaFuncAttributePreferredSharedMemoryCarveout, carve);
+    cudaError_t e = carveout<4, 1, false>();
+    if (e == cudaSuccess) e = carveout<6, 1, false>();
+    if (e == cudaSuccess) e = carveout<4, 0, false>();
+    if (e == cudaSuccess) e = carveout<6, 0, false>();
+    if (e == cudaSuccess) e = carveout<4, 1, true>();
+    if (e == cudaSuccess) e = carveout<6, 1, true>();
+    if (e == cudaSuccess) e = carveout<4, 0, true>();
+    if (e == cudaSuccess) e = carveout<6, 0, true>();
     return e;
 }
 
@@ -202,18 +241,14 @@ cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    const float *Y = plan.ws.Y;
     // y_dev is 16-byte aligned; rows of an even W keep 8-byte alignment for every tile
     if (g.m == 4) {
-        if (g.W % 4 == 0)
-            return cudaLaunchKernelEx(&cfg, output_transform_kernel<4, 2>, Y, y_dev, g, plan.tables);
-        if (g.W % 2 == 0)
-            return cudaLaunchKernelEx(&cfg, output_transform_kernel<4, 1>, Y, y_dev, g, plan.tables);
-        return cudaLaunchKernelEx(&cfg, output_transform_kernel<4, 0>, Y, y_dev, g, plan.tables);
+        if (g.W % 4 == 0) return launch_variant<4, 2>(cfg, plan, y_dev);
+        if (g.W % 2 == 0) return launch_variant<4, 1>(cfg, plan, y_dev);
+        return launch_variant<4, 0>(cfg, plan, y_dev);
     }
-    if (g.W % 2 == 0)
-        return cudaLaunchKernelEx(&cfg, output_transform_kernel<6, 1>, Y, y_dev, g, plan.tables);
-    return cudaLaunchKernelEx(&cfg, output_transform_kernel<6, 0>, Y, y_dev, g, plan.tables);
+    if (g.W % 2 == 0) return launch_variant<6, 1>(cfg, plan, y_dev);
+    return launch_variant<6, 0>(cfg, plan, y_dev);
 }
 
 }  // namespace wfq

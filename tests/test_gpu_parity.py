@@ -107,6 +107,41 @@ def test_negative_and_standard_scales():
     _check(L, (x, w, np.array(learned["SB"], np.float32), np.array(learned["SG"], np.float32)))
 
 
+@pytest.mark.parametrize("m,H,W", [(4, 16, 16), (4, 9, 14), (4, 7, 7), (6, 12, 12), (6, 13, 11)],
+                         ids=["f43_w16", "f43_w14", "f43_w7", "f63_w12", "f63_w11"])
+def test_bias_and_activation_epilogue(m, H, W):
+    """y = act(conv + bias) fused into the output transform, every store variant; the
+    setting can be changed and cleared between calls on one plan."""
+    import torch
+    from oracle import oracle as orc
+    from paper_2412_19867_b200 import binding as b
+    from tests import gpu_util as gu
+    L = Layer(2, 64, 40, H, W, m, 32, "f16", "silu_outlier", "kaiming_chan", 9, 2, 50 + W)
+    conv, (x, w, sB, sG) = gu.make_conv(L)
+    xd = torch.from_numpy(x).to("cuda:0")
+    ref = orc.wfq(x, w, L.m, L.gs, sB, sG).y
+    scale = float(np.max(np.abs(ref)))
+    rng = np.random.default_rng(7)
+    bias = (rng.standard_normal(L.K) * 0.5 * scale).astype(np.float32)
+    bd = torch.from_numpy(bias).to("cuda:0")
+    for act_id, act in ((b.WFQ_ACT_RELU, "relu"), (b.WFQ_ACT_SILU, "silu"), (b.WFQ_ACT_NONE, "none")):
+        for use_bias in (True, False):
+            if act == "none" and not use_bias:
+                continue
+            conv.set_epilogue(bd if use_bias else None, act_id)
+            y = conv.forward(xd).cpu().numpy()
+            conv.check_status()
+            want = orc.epilogue(ref, bias if use_bias else None, act)
+            err = float(np.max(np.abs(y - want))) / scale
+            assert err <= gu.FINAL_TOL, (act, use_bias, err)
+    conv.set_epilogue(None, b.WFQ_ACT_NONE)
+    y = conv.forward(xd).cpu().numpy()
+    assert float(np.max(np.abs(y - ref))) / scale <= gu.FINAL_TOL
+    with pytest.raises(b.WfqError):
+        b.wfq_plan_set_epilogue(conv.plan, None, 7)
+    conv.close()
+
+
 def test_host_buffer_entry_point_matches_device_one():
     import torch
     from tests.gpu_util import make_conv

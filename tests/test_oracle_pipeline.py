@@ -270,3 +270,21 @@ def test_workload_generators_are_seeded_and_shaped():
         np.testing.assert_array_equal(u, v)
     assert a[0].dtype == np.float16 and a[0].shape == (2, 1280, 16, 16)
     assert a[1].shape == (1280, 1280, 3, 3) and a[2].shape == (6,)
+
+
+def test_epilogue_hand_values():
+    """Bias per output channel, then ReLU / SiLU: hand-computed values (silu(1) = 1 / (1 + 1/e),
+    silu(0) = 0, silu(-t) = silu(t) - t)."""
+    y = np.array([[[[1.0, -2.0]], [[0.5, 0.0]]]])          # [1][2][1][2]
+    bias = np.array([0.0, -0.5])
+    np.testing.assert_allclose(orc.epilogue(y, bias, "none"), [[[[1.0, -2.0]], [[0.0, -0.5]]]])
+    np.testing.assert_allclose(orc.epilogue(y, bias, "relu"), [[[[1.0, 0.0]], [[0.0, 0.0]]]])
+    s = orc.epilogue(y, None, "silu")
+    e = 2.718281828459045
+    np.testing.assert_allclose(s[0, 0, 0, 0], 1.0 / (1.0 + 1.0 / e), rtol=1e-15)
+    assert s[0, 1, 0, 1] == 0.0
+    np.testing.assert_allclose(s[0, 0, 0, 1], 2.0 / (1.0 + e * e) * e * e - 2.0, rtol=1e-13)
+    t = np.linspace(-5, 5, 11).reshape(1, 1, 1, 11)
+    np.testing.assert_allclose(orc.epilogue(-t, None, "silu"), orc.epilogue(t, None, "silu") - t, atol=1e-15)
+    with pytest.raises(ValueError):
+        orc.epilogue(y, None, "gelu")
