@@ -121,6 +121,26 @@ wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype);
 wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_activation_t act);
 
 /*
+ * The paper's fully quantized transforms (Section 4.1), off by default.
+ *   quant_input  1: the input transform runs on integer codes (Eq. quant-B): x is quantized to 8
+ *                bits with one scale per (tile, channel group) over the group's n x n patches,
+ *                S_B V_B to 8 bits with one scale, the two matrix products are integer products
+ *                and the result times s_qB^2 s_qx is what the group quantizer of the contraction
+ *                sees.  0: floating-point input transform.
+ *   y_mode       WFQ_Y_FP32: floating-point output transform; WFQ_Y_TILE / WFQ_Y_ROW: the output
+ *                transform runs on integer codes (Eq. quant-y) with V_A S_A quantized to 8 bits
+ *                with one scale and Y with one scale per (tile, output channel), or with one
+ *                scale per row of the n x n matrix and, after the first product, one per column
+ *                (Section 3.2: Y needs a scale per tile or per row / column).
+ * With an integer output transform the scale vectors given to wfq_prepare_filters change the
+ * result (this is where the paper's learned scales act); with the floating-point transforms they
+ * are numerically neutral.  Group sizes: multiples of 32 up to 256.  Host only; takes effect from
+ * the next forward call.  These kernels are reference-speed implementations.
+ */
+typedef enum { WFQ_Y_FP32 = 0, WFQ_Y_TILE = 1, WFQ_Y_ROW = 2 } wfq_y_quant_t;
+wfq_status_t wfq_plan_set_full_quant(wfq_plan_t *plan, int quant_input, wfq_y_quant_t y_mode);
+
+/*
  * Bytes of caller-owned device scratch the plan needs (Xq + sX + Y, each region
  * 1024-byte aligned).  Returns 0 for a NULL plan.
  */

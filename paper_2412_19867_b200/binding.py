@@ -16,6 +16,7 @@ WFQ_ERR_NOT_PREPARED, WFQ_ERR_CUDA, WFQ_ERR_TIMEOUT, WFQ_ERR_SCRATCH_TOO_SMALL =
 WFQ_STATIC_SCRATCH_FLOATS = 4 * 1024 * 1024
 WFQ_F32, WFQ_F16 = 0, 1
 WFQ_ACT_NONE, WFQ_ACT_RELU, WFQ_ACT_SILU = 0, 1, 2
+WFQ_Y_FP32, WFQ_Y_TILE, WFQ_Y_ROW = 0, 1, 2
 WFQ_BUF_XQ, WFQ_BUF_SX, WFQ_BUF_WQ, WFQ_BUF_SW, WFQ_BUF_Y, WFQ_BUF_STATUS = range(6)
 WFQ_DEBUG_WAIT_CYCLES, WFQ_DEBUG_SKIP_INPUT_ITEM, WFQ_DEBUG_INPUT_TRANSFORM_KERNEL = range(3)
 WFQ_DEBUG_SKIP_GEMM_STAGE = 3
@@ -28,7 +29,7 @@ EXPORTS = [
     "wfq_output_transform", "wfq_debug_gemm_acc32", "wfq_debug_get",
     "wfq_check_device_status", "wfq_plan_destroy", "wfq_status_string", "wfq_version",
     "wfq_quantize_filters_static", "wfq_plan_set_debug_option", "wfq_debug_int8_mma_rate",
-    "wfq_plan_set_epilogue",
+    "wfq_plan_set_epilogue", "wfq_plan_set_full_quant",
 ]
 
 _lib = None
@@ -67,6 +68,7 @@ def load():
     lib.wfq_plan_destroy.argtypes = [vp]
     lib.wfq_quantize_filters_static.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
     lib.wfq_plan_set_epilogue.argtypes = [vp, vp, ci]
+    lib.wfq_plan_set_full_quant.argtypes = [vp, ci, ci]
     lib.wfq_plan_set_debug_option.argtypes = [vp, ci, ctypes.c_longlong]
     lib.wfq_debug_int8_mma_rate.argtypes = [vp, ci, ci, ctypes.POINTER(ctypes.c_longlong), vp]
     lib.wfq_status_string.argtypes = [ci]
@@ -111,6 +113,10 @@ def wfq_plan_set_input_dtype(plan, dtype):
 
 def wfq_plan_set_epilogue(plan, bias_dev, act=WFQ_ACT_NONE):
     _check(load().wfq_plan_set_epilogue(plan, bias_dev, act), "wfq_plan_set_epilogue")
+
+
+def wfq_plan_set_full_quant(plan, quant_input, y_mode):
+    _check(load().wfq_plan_set_full_quant(plan, int(quant_input), y_mode), "wfq_plan_set_full_quant")
 
 
 def wfq_plan_workspace_bytes(plan):

@@ -59,7 +59,8 @@ wfq_status_t bind_device(wfq_plan *plan)
         std::lock_guard<std::mutex> lock(g_setup_mutex);
         if (!g_device_ready[dev]) {
             if (wfq::setup_input_transform() != cudaSuccess || wfq::setup_input_transform_tc() != cudaSuccess ||
-                wfq::setup_gemm() != cudaSuccess || wfq::setup_output_transform() != cudaSuccess)
+                wfq::setup_gemm() != cudaSuccess || wfq::setup_output_transform() != cudaSuccess ||
+                wfq::setup_full_quant() != cudaSuccess)
                 return WFQ_ERR_CUDA;
             g_device_ready[dev] = true;
         }
@@ -204,6 +205,19 @@ wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_
 
 size_t wfq_plan_workspace_bytes(const wfq_plan_t *plan) { return plan ? plan->ws.total : 0; }
 
+wfq_status_t wfq_plan_set_full_quant(wfq_plan_t *plan, int quant_input, wfq_y_quant_t y_mode)
+{
+    if (!plan) return WFQ_ERR_INVALID_ARG;
+    if (quant_input != 0 && quant_input != 1) return WFQ_ERR_INVALID_ARG;
+    if (y_mode != WFQ_Y_FP32 && y_mode != WFQ_Y_TILE && y_mode != WFQ_Y_ROW) return WFQ_ERR_INVALID_ARG;
+    if (quant_input && (plan->geo.gs % 32 != 0 || plan->geo.gs > 256)) return WFQ_ERR_UNSUPPORTED;
+    plan->fq_input = quant_input != 0;
+    plan->fq_output = (int)y_mode;
+    for (int i = 0; i < 2; ++i)
+        if (plan->sub[i]) { plan->sub[i]->fq_input = plan->fq_input; plan->sub[i]->fq_output = plan->fq_output; }
+    return WFQ_OK;
+}
+
 wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t bytes)
 {
     if (!plan || !dev_ptr) return WFQ_ERR_INVALID_ARG;
@@ -284,6 +298,7 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
     plan->tmap_wq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_wq, plan->Wq, g.C, g.K, g.P,
                                                plan->gemm_swap ? wfq::gemm_block_m() : plan->gemm_bn);
     if (!plan->tmap_wq_ok) return WFQ_ERR_CUDA;
+    wfq::build_full_quant_tables(*plan);
     plan->prepared = true;
     return WFQ_OK;
 }
@@ -293,6 +308,7 @@ wfq_status_t wfq_input_transform_quantize(wfq_plan_t *plan, const void *x_dev, v
     wfq_status_t s = ready_to_run(plan);
     if (s != WFQ_OK) return s;
     if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 3u)) return WFQ_ERR_INVALID_ARG;
+    if (plan->fq_input) return cuda_status(wfq::launch_input_transform_int(*plan, x_dev, as_stream(stream)));
     return cuda_status(wfq::launch_input_transform(*plan, x_dev, as_stream(stream)));
 }
 
@@ -328,6 +344,7 @@ wfq_status_t wfq_output_transform(wfq_plan_t *plan, float *y_dev, void *stream)
     wfq_status_t s = ready_to_run(plan);
     if (s != WFQ_OK) return s;
     if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 15u)) return WFQ_ERR_INVALID_ARG;
+    if (plan->fq_output) return cuda_status(wfq::launch_output_transform_int(*plan, y_dev, as_stream(stream)));
     return cuda_status(wfq::launch_output_transform(*plan, y_dev, as_stream(stream), false));
 }
 
@@ -339,9 +356,12 @@ wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev,
         (reinterpret_cast<uintptr_t>(y_dev) & 15u))
         return WFQ_ERR_INVALID_ARG;
     cudaStream_t st = as_stream(stream);
-    cudaError_t e = wfq::launch_input_transform(*plan, x_dev, st);
+    cudaError_t e = plan->fq_input ? wfq::launch_input_transform_int(*plan, x_dev, st)
+                                   : wfq::launch_input_transform(*plan, x_dev, st);
     if (e == cudaSuccess) e = wfq::launch_gemm(*plan, nullptr, st, true);
-    if (e == cudaSuccess) e = wfq::launch_output_transform(*plan, y_dev, st, true);
+    if (e == cudaSuccess)
+        e = plan->fq_output ? wfq::launch_output_transform_int(*plan, y_dev, st)
+                            : wfq::launch_output_transform(*plan, y_dev, st, true);
     return cuda_status(e);
 }
 
@@ -385,6 +405,7 @@ static wfq_status_t setup_host_pipeline(wfq_plan *plan)
         q->tmap_wq = plan->tmap_wq; q->tmap_wq_ok = plan->tmap_wq_ok;
         q->wait_cycles = plan->wait_cycles;
         q->bias = plan->bias; q->act = plan->act;
+        q->fq_input = plan->fq_input; q->fq_output = plan->fq_output; q->fq = plan->fq;
         q->prepared = true;
         if (!plan->host_stream[s] &&
             cudaStreamCreateWithFlags(&plan->host_stream[s], cudaStreamNonBlocking) != cudaSuccess)

@@ -51,6 +51,15 @@ struct ScaleTables {
     float out_scale[kMaxP];  // sA_i*sA_j: applied before the output transform
 };
 
+// Codes and scales of the two transform matrices for the fully quantized transforms
+// (Eqs. quant-B and quant-y), built on the host from the plan's scale vectors.
+struct FullQuantTables {
+    int BTq[kMaxN * kMaxN];   // Q(S_B V_B / s_qB), [i][a], n x n
+    int ATq[kMaxN * kMaxN];   // Q(V_A S_A / s_qA), [u][i], m x n at row pitch n
+    double sqB2;              // s_qB^2
+    double sqA;               // s_qA
+};
+
 // Launch parameters of the cp.async input-transform kernel (any dtype, any shape),
 // computed once per plan.
 struct K1Params {
@@ -116,6 +125,9 @@ struct wfq_plan {
     long long wait_cycles = 2000000000LL;   // limit of every device-side wait (~1 s)
     int debug_skip_item = -1;  // >= 0: the input transform's producer skips this work item
     int debug_skip_gemm_stage = -1;   // >= 0: the contraction's producer (CTA 0) skips this stage
+    bool fq_input = false;     // input transform on integer codes (Eq. quant-B)
+    int fq_output = 0;         // output transform: 0 fp32, 1 integer with one scale of Y per tile, 2 per row / column
+    wfq::FullQuantTables fq;   // valid once the filters are prepared
     int k1_choice = 0;         // input-transform kernel: 0 automatic, 1 cp.async, 2 tensor cores where they apply
 
     CUtensorMap tmap_xq;       // Xq as (C, T, P) bytes, 128B-swizzled boxes
@@ -161,6 +173,10 @@ bool encode_tmap(CUtensorMap *map, CUtensorMapDataType dtype, int rank, const vo
                  const unsigned *box, CUtensorMapSwizzle swizzle);
 cudaError_t launch_gemm(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t stream, bool pdl);
 cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStream_t stream, bool pdl);
+void build_full_quant_tables(wfq_plan &plan);
+cudaError_t setup_full_quant();
+cudaError_t launch_input_transform_int(const wfq_plan &plan, const void *x_dev, cudaStream_t stream);
+cudaError_t launch_output_transform_int(const wfq_plan &plan, float *y_dev, cudaStream_t stream);
 cudaError_t launch_mma_peak(const wfq_plan &plan, int n_cols, int mmas, cudaStream_t stream);
 
 // Builds a 3-D byte tensor map (inner extent `inner`, rows, planes) with a

@@ -113,6 +113,8 @@ def _activations(rng, layer):
         z = rng.standard_normal(shape)
         x = z / (1.0 + np.exp(-z))
         x = np.where(rng.random(shape) < 0.005, 50.0 * x, x)
+    elif layer.act == "gauss":
+        x = rng.standard_normal(shape)          # the random-noise inputs of the data-free setting
     elif layer.act == "zeros":
         x = np.zeros(shape)
     else:
