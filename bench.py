@@ -279,7 +279,7 @@ def select_layers(wl, cfg, only_layer=None):
 class Workload:
     """The layers of one configuration: plans, device tensors, and the step as a CUDA graph."""
 
-    def __init__(self, cfg, only_layer, dev, stream, flush, use_graph=True, k1_kernel=0):
+    def __init__(self, cfg, only_layer, dev, stream, flush, use_graph=True, k1_kernel=0, full_quant=None):
         import torch
         from paper_2412_19867_b200 import binding as b
         from paper_2412_19867_b200 import workloads as wl
@@ -293,6 +293,8 @@ class Workload:
             conv.prepare(torch.from_numpy(w).to(dev), list(sB), list(sG))
             if k1_kernel:
                 b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, k1_kernel)
+            if full_quant is not None:      # (integer input transform, scale of Y: 1 per tile, 2 per row / column)
+                b.wfq_plan_set_full_quant(conv.plan, full_quant[0], full_quant[1])
             self.convs.append(conv)
             self.xs.append(torch.from_numpy(x).to(dev))
             self.ys.append(torch.empty((L.N, L.K, L.H, L.W), dtype=torch.float32, device=dev))
@@ -442,6 +444,41 @@ class Workload:
                     worst, worst_layer = err, L.name
         return {"checked": True, "against": "CPU oracle, sampled tiles and output channels of every layer",
                 "worst_rel_err": worst, "worst_layer": worst_layer, "tolerance": 2e-3, "ok": worst <= 2e-3,
+                "int8_code_mismatch_rate": mism / max(ncodes, 1), "codes_compared": ncodes}
+
+    def parity_full_quant(self, y_scale, tiles_per_layer=6, channels=12):
+        """The fully quantized pipeline's outputs against the oracle's on sampled tiles and
+        output channels: relative L2 distance over the sample (a code of Y that flips through
+        the fp32 accumulation order of Y moves one tile by a quantization step, so there is
+        no element-wise bar) and the mismatch rate of the int8 codes (bit exact by design)."""
+        import numpy as np
+        from oracle import full_quant as fq
+        from oracle import oracle as orc
+        b, torch = self.b, self.torch
+        num = den = 0.0
+        mism = ncodes = 0
+        for L, conv, (x, w, sB, sG), y in zip(self.layers, self.convs, self.tensors, self.ys):
+            yh = y.cpu().numpy()
+            rng = np.random.default_rng(L.seed + 17)
+            T = conv.T
+            tiles = np.unique(np.concatenate([[0, T - 1], rng.integers(0, T, tiles_per_layer)]))
+            ks = np.unique(np.concatenate([[0, L.K - 1], rng.integers(0, L.K, channels)]))
+            ref = fq.wfq_full(x, w[ks], L.m, L.gs, sB, sG, tiles=tiles, quant_input=True, quant_output=True,
+                              y_scale=y_scale)
+            xq = conv.buffer(b.WFQ_BUF_XQ)[:, torch.from_numpy(tiles).to(self.dev)].cpu().numpy()
+            mism += int(np.count_nonzero(xq != ref.Xq))
+            ncodes += xq.size
+            geo = orc.geometry(L.N, L.H, L.W, L.m)
+            for i, t in enumerate(tiles):
+                tw, th, img = t % geo.TW, (t // geo.TW) % geo.TH, t // (geo.TW * geo.TH)
+                hh, ww = min(L.m, L.H - th * L.m), min(L.m, L.W - tw * L.m)
+                got = yh[img][ks][:, th * L.m:th * L.m + hh, tw * L.m:tw * L.m + ww]
+                want = ref.ytile[i][:, :hh, :ww]
+                num += float(np.sum((got - want) ** 2))
+                den += float(np.sum(want ** 2))
+        rel = (num / max(den, 1e-300)) ** 0.5
+        return {"against": "CPU oracle of the fully quantized pipeline, sampled tiles and output channels",
+                "rel_l2": rel, "tolerance": 1e-2, "ok": rel <= 1e-2,
                 "int8_code_mismatch_rate": mism / max(ncodes, 1), "codes_compared": ncodes}
 
     def close(self):
@@ -676,6 +713,33 @@ def run_wfq(args):
             except Exception as exc:
                 per_config[f"cfg{cfg}"] = {"error": repr(exc)}
 
+    # ---- the fully quantized transforms (Section 4.1) on the UNet block, reported beside ----
+    full_quant = None
+    if rank == 0 and world == 1 and not args.no_extras and args.only_layer is None:
+        full_quant = {}
+        for label, mode, y_scale in (("y_per_tile", 1, "tile"), ("y_per_row_column", 2, "row")):
+            try:
+                w3 = Workload(4, None, dev, stream, flush, use_graph=not args.no_graph, full_quant=(1, mode))
+                for _ in range(3):
+                    flush.zero_()
+                    w3.step()
+                torch.cuda.synchronize(dev)
+                ms = [statistics.median(w3.timed_replays(reps)) for _ in range(10)]
+                s3, _, _ = w3.summary(statistics.mean(ms), w3.kernel_split(10), peak)
+                flush.zero_()
+                w3.step()
+                torch.cuda.synchronize(dev)
+                full_quant[label] = {"workload": s3["workload"], "value": s3["value"], "unit": UNIT,
+                                     "us_per_step": s3["us_per_step"], "kernels": s3["kernels"],
+                                     "us_per_layer": s3["us_per_layer"], "parity": w3.parity_full_quant(y_scale),
+                                     "note": "integer input and output transforms (Eqs. quant-B, quant-y), "
+                                             "reference-speed kernels; same contraction kernel"}
+                w3.close()
+                del w3
+                torch.cuda.empty_cache()
+            except Exception as exc:
+                full_quant[label] = {"error": repr(exc)}
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         o, s, sample, cores = oracle_time_sample(layers, tensors, args.cpu_seconds)
@@ -694,7 +758,7 @@ def run_wfq(args):
                            "parallelism": "replicas" if world > 1 else "single GPU"},
                 "timing": timing, "us_per_layer": head["us_per_layer"], "wall_s_timed_region": wall,
                 "warm": warm, "sustained": sustained, "roofline": roofline, "contraction": contraction,
-                "parity": parity, "per_config": per_config, "cpu_baseline": cpu, "e2e": e2e,
+                "parity": parity, "per_config": per_config, "full_quant": full_quant, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": 3 * len(layers) * args.steps * reps, "clocks": clocks}
         print(json.dumps(line), flush=True)
     if world > 1:
