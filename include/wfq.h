@@ -121,6 +121,14 @@ wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype);
 wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_activation_t act);
 
 /*
+ * Element type of the output y: WFQ_F32 (default) or WFQ_F16.  With WFQ_F16 the output transform
+ * rounds each result once to fp16 (after bias and activation) and `y_nkhw_dev` / `y_host` of the
+ * forward calls point at fp16 storage of the same [N][K][H][W] shape (the parameters keep their
+ * `float *` type; alignment requirements are unchanged).  Host only.
+ */
+wfq_status_t wfq_plan_set_output_dtype(wfq_plan_t *plan, wfq_dtype_t dtype);
+
+/*
  * The paper's fully quantized transforms (Section 4.1), off by default.
  *   quant_input  1: the input transform runs on integer codes (Eq. quant-B): x is quantized to 8
  *                bits with one scale per (tile, channel group) over the group's n x n patches,

@@ -29,7 +29,7 @@ EXPORTS = [
     "wfq_output_transform", "wfq_debug_gemm_acc32", "wfq_debug_get",
     "wfq_check_device_status", "wfq_plan_destroy", "wfq_status_string", "wfq_version",
     "wfq_quantize_filters_static", "wfq_plan_set_debug_option", "wfq_debug_int8_mma_rate",
-    "wfq_plan_set_epilogue", "wfq_plan_set_full_quant",
+    "wfq_plan_set_epilogue", "wfq_plan_set_full_quant", "wfq_plan_set_output_dtype",
 ]
 
 _lib = None
@@ -69,6 +69,7 @@ def load():
     lib.wfq_quantize_filters_static.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
     lib.wfq_plan_set_epilogue.argtypes = [vp, vp, ci]
     lib.wfq_plan_set_full_quant.argtypes = [vp, ci, ci]
+    lib.wfq_plan_set_output_dtype.argtypes = [vp, ci]
     lib.wfq_plan_set_debug_option.argtypes = [vp, ci, ctypes.c_longlong]
     lib.wfq_debug_int8_mma_rate.argtypes = [vp, ci, ci, ctypes.POINTER(ctypes.c_longlong), vp]
     lib.wfq_status_string.argtypes = [ci]
@@ -113,6 +114,10 @@ def wfq_plan_set_input_dtype(plan, dtype):
 
 def wfq_plan_set_epilogue(plan, bias_dev, act=WFQ_ACT_NONE):
     _check(load().wfq_plan_set_epilogue(plan, bias_dev, act), "wfq_plan_set_epilogue")
+
+
+def wfq_plan_set_output_dtype(plan, dtype):
+    _check(load().wfq_plan_set_output_dtype(plan, dtype), "wfq_plan_set_output_dtype")
 
 
 def wfq_plan_set_full_quant(plan, quant_input, y_mode):
@@ -238,6 +243,11 @@ class Conv:
         with torch.cuda.device(self.device):
             wfq_prepare_filters(self.plan, w.data_ptr(), sB, sG, sA, self._stream())
 
+    def set_output_dtype(self, dtype):
+        """"f32" (default) or "f16": element type of the tensors forward() returns or fills."""
+        self.out_dtype = dtype
+        wfq_plan_set_output_dtype(self.plan, WFQ_F16 if dtype == "f16" else WFQ_F32)
+
     def set_epilogue(self, bias=None, act=WFQ_ACT_NONE):
         """bias: fp32 CUDA tensor [K] or None; kept alive by this object."""
         if bias is not None:
@@ -251,8 +261,10 @@ class Conv:
         N, C, K, H, W = self.shape
         assert x.is_cuda and x.is_contiguous() and tuple(x.shape) == (N, C, H, W)
         assert x.dtype == (torch.float16 if self.in_dtype == "f16" else torch.float32)
+        ydt = torch.float16 if getattr(self, "out_dtype", "f32") == "f16" else torch.float32
         if y is None:
-            y = torch.empty((N, K, H, W), dtype=torch.float32, device=self.device)
+            y = torch.empty((N, K, H, W), dtype=ydt, device=self.device)
+        assert y.dtype == ydt and y.is_contiguous() and tuple(y.shape) == (N, K, H, W)
         with torch.cuda.device(self.device):
             wfq_conv_forward(self.plan, x.data_ptr(), y.data_ptr(), self._stream())
         return y

@@ -205,6 +205,16 @@ wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_
 
 size_t wfq_plan_workspace_bytes(const wfq_plan_t *plan) { return plan ? plan->ws.total : 0; }
 
+wfq_status_t wfq_plan_set_output_dtype(wfq_plan_t *plan, wfq_dtype_t dtype)
+{
+    if (!plan || (dtype != WFQ_F32 && dtype != WFQ_F16)) return WFQ_ERR_INVALID_ARG;
+    plan->out_half = dtype == WFQ_F16;
+    plan->host_chunks = 0;         // chunk sizes of the host-buffer path depend on the output bytes
+    for (int i = 0; i < 2; ++i)
+        if (plan->sub[i]) plan->sub[i]->out_half = plan->out_half;
+    return WFQ_OK;
+}
+
 wfq_status_t wfq_plan_set_full_quant(wfq_plan_t *plan, int quant_input, wfq_y_quant_t y_mode)
 {
     if (!plan) return WFQ_ERR_INVALID_ARG;
@@ -404,7 +414,7 @@ static wfq_status_t setup_host_pipeline(wfq_plan *plan)
         q->tables = plan->tables;
         q->tmap_wq = plan->tmap_wq; q->tmap_wq_ok = plan->tmap_wq_ok;
         q->wait_cycles = plan->wait_cycles;
-        q->bias = plan->bias; q->act = plan->act;
+        q->bias = plan->bias; q->act = plan->act; q->out_half = plan->out_half;
         q->fq_input = plan->fq_input; q->fq_output = plan->fq_output; q->fq = plan->fq;
         q->prepared = true;
         if (!plan->host_stream[s] &&
@@ -426,11 +436,12 @@ wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *
     if (!x_host || !y_host) return WFQ_ERR_INVALID_ARG;
     const wfq::Geometry &g = plan->geo;
     const size_t xb = (size_t)g.N * g.C * g.H * g.W * in_elem_bytes(plan);
-    const size_t yb = (size_t)g.N * g.K * g.H * g.W * sizeof(float);
+    const size_t yb = (size_t)g.N * g.K * g.H * g.W * (plan->out_half ? 2 : sizeof(float));
     cudaError_t e;
     if (!plan->x_stage && (e = cudaMalloc(&plan->x_stage, (size_t)g.N * g.C * g.H * g.W * 4)) != cudaSuccess)
         return cuda_status(e);
-    if (!plan->y_stage && (e = cudaMalloc(&plan->y_stage, yb)) != cudaSuccess) return cuda_status(e);
+    if (!plan->y_stage && (e = cudaMalloc(&plan->y_stage, (size_t)g.N * g.K * g.H * g.W * sizeof(float))) != cudaSuccess)
+        return cuda_status(e);
     cudaStream_t st = as_stream(stream);
 
     if (plan->host_chunks == 0) plan->host_chunks = pick_host_chunks(plan, xb, yb);
@@ -448,7 +459,7 @@ wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *
         for (int c = 0; c < chunks && err == WFQ_OK; ++c) {
             cudaStream_t cs = plan->host_stream[c & 1];
             char *xd = static_cast<char *>(plan->x_stage) + (size_t)c * xc;
-            float *yd = plan->y_stage + (size_t)c * (yc / sizeof(float));
+            float *yd = reinterpret_cast<float *>(reinterpret_cast<char *>(plan->y_stage) + (size_t)c * yc);
             if (cudaMemcpyAsync(xd, static_cast<const char *>(x_host) + (size_t)c * xc, xc,
                                 cudaMemcpyHostToDevice, cs) != cudaSuccess) {
                 err = WFQ_ERR_CUDA;

@@ -139,7 +139,7 @@ __global__ void input_transform_int_kernel(const Tin *__restrict__ x, int8_t *__
 template <int M, int MODE>
 __global__ void __launch_bounds__(128)
 output_transform_int_kernel(const float *__restrict__ Y, float *__restrict__ y, Geometry g,
-                            FullQuantTables tab, const float *__restrict__ bias, int act)
+                            FullQuantTables tab, const float *__restrict__ bias, int act, int out_half)
 {
     constexpr int NN = M + 2;
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
@@ -235,7 +235,8 @@ output_transform_int_kernel(const float *__restrict__ Y, float *__restrict__ y, 
                 float r = (float)out[u][c] + bk;
                 if (act == 1) r = fmaxf(r, 0.f);
                 else if (act == 2) r = r * __frcp_rn(1.f + __expf(-r));
-                dst[(size_t)u * g.W + c] = r;
+                if (out_half) reinterpret_cast<__half *>(y)[(dst - y) + (size_t)u * g.W + c] = __float2half_rn(r);
+                else dst[(size_t)u * g.W + c] = r;
             }
 }
 
@@ -338,11 +339,11 @@ cudaError_t launch_output_transform_int(const wfq_plan &plan, float *y_dev, cuda
     const dim3 grid((unsigned)((g.T + 127) / 128), (unsigned)g.K), block(128);
     const float *Y = plan.ws.Y;
     if (plan.fq_output == 1) {
-        if (g.m == 4) output_transform_int_kernel<4, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act);
-        else output_transform_int_kernel<6, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act);
+        if (g.m == 4) output_transform_int_kernel<4, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
+        else output_transform_int_kernel<6, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
     } else {
-        if (g.m == 4) output_transform_int_kernel<4, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act);
-        else output_transform_int_kernel<6, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act);
+        if (g.m == 4) output_transform_int_kernel<4, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
+        else output_transform_int_kernel<6, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
     }
     return cudaGetLastError();
 }

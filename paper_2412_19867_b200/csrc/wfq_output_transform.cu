@@ -3,6 +3,8 @@
 // Y[P][K][Tp] are 128-byte coalesced; the m-float row segments of neighbouring tiles are
 // contiguous in y[N][K][H][W] and are written in whole sectors.  P*4 bytes read
 // and m*m*4 bytes written per thread against ~150 flops.
+#include <cuda_fp16.h>
+
 #include "wfq_internal.h"
 #include "wfq_ptx.cuh"
 
@@ -68,8 +70,10 @@ __device__ __forceinline__ void epilogue(float (&o)[M], float bias, int act)
 template <int M, int STORE, bool EPI>
 __global__ void __launch_bounds__(128, M == 6 ? (EPI ? 6 : 7) : 8)
 output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geometry g,
-                        ScaleTables tab, const float *__restrict__ bias, int act)
+                        ScaleTables tab, const float *__restrict__ bias, int act, int out_half)
 {
+    // fp16 output (epilogue variants only): y points at __half storage of the same shape
+    [[maybe_unused]] __half *yh = reinterpret_cast<__half *>(y);
     constexpr int NN = M + 2;
     constexpr int TT = 128;                       // tiles per CTA
     __shared__ __align__(16) float out_s[STORE != 2 ? M * TT * M : 1];   // [u][tile][v]
@@ -146,8 +150,11 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
                     const int f = threadIdx.x + i * TT;
                     const int tj = f / M, v1 = f - tj * M;
                     const int lim = tile_lim[tj];
-                    if (u < (lim >> 4) && v1 < (lim & 15))
-                        y[(size_t)tile_base[tj] + (size_t)u * g.W + v1] = row[f];
+                    if (u < (lim >> 4) && v1 < (lim & 15)) {
+                        const size_t off = (size_t)tile_base[tj] + (size_t)u * g.W + v1;
+                        if (EPI && out_half) yh[off] = __float2half_rn(row[f]);
+                        else y[off] = row[f];
+                    }
                 }
             }
             return;
@@ -162,12 +169,16 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
                 const int q = threadIdx.x + i * TT;
                 const int tj = q / PPT, v2 = 2 * (q - tj * PPT);
                 const int lim = tile_lim[tj];
-                if (u < (lim >> 4) && v2 < (lim & 15))      // W even: both columns or none
-                    *reinterpret_cast<float2 *>(y + (size_t)tile_base[tj] + (size_t)u * g.W + v2) = row[q];
+                if (u < (lim >> 4) && v2 < (lim & 15)) {    // W even: both columns or none
+                    const size_t off = (size_t)tile_base[tj] + (size_t)u * g.W + v2;
+                    if (EPI && out_half) *reinterpret_cast<__half2 *>(yh + off) = __float22half2_rn(row[q]);
+                    else *reinterpret_cast<float2 *>(y + off) = row[q];
+                }
             }
         }
     } else {
         float *row = y + base;
+        __half *rowh = yh + base;
         const bool full_w = (w0 + M <= g.W);
         const float bk = (EPI && bias) ? __ldg(bias + k) : 0.f;
 #pragma unroll
@@ -176,7 +187,17 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
             at_1d<M>(tmp[u], o);
             if constexpr (EPI) epilogue<M>(o, bk, act);
             if (h0 + u < g.H) {
-                if (full_w) {
+                if (EPI && out_half) {
+                    if (full_w) {
+                        const __half2 lo = __floats2half2_rn(o[0], o[1]), hi = __floats2half2_rn(o[2], o[3]);
+                        *reinterpret_cast<uint2 *>(rowh) = make_uint2(*reinterpret_cast<const uint32_t *>(&lo),
+                                                                      *reinterpret_cast<const uint32_t *>(&hi));
+                    } else {
+#pragma unroll
+                        for (int v2 = 0; v2 < M; ++v2)
+                            if (w0 + v2 < g.W) rowh[v2] = __float2half_rn(o[v2]);
+                    }
+                } else if (full_w) {
                     *reinterpret_cast<float4 *>(row) = make_float4(o[0], o[1], o[2], o[3]);
                 } else {
 #pragma unroll
@@ -185,6 +206,7 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
                 }
             }
             row += g.W;
+            rowh += g.W;
         }
     }
 }
@@ -204,11 +226,12 @@ template <int M, int STORE>
 cudaError_t launch_variant(const cudaLaunchConfig_t &cfg, const wfq_plan &plan, float *y_dev)
 {
     const float *Y = plan.ws.Y;
-    if (plan.bias || plan.act)
+    const int out_half = plan.out_half ? 1 : 0;
+    if (plan.bias || plan.act || out_half)
         return cudaLaunchKernelEx(&cfg, output_transform_kernel<M, STORE, true>, Y, y_dev, plan.geo, plan.tables,
-                                  plan.bias, plan.act);
+                                  plan.bias, plan.act, out_half);
     return cudaLaunchKernelEx(&cfg, output_transform_kernel<M, STORE, false>, Y, y_dev, plan.geo, plan.tables,
-                              plan.bias, plan.act);
+                              plan.bias, plan.act, out_half);
 }
 
 }  // namespace

@@ -142,6 +142,37 @@ def test_bias_and_activation_epilogue(m, H, W):
     conv.close()
 
 
+@pytest.mark.parametrize("m,H,W", [(4, 16, 16), (4, 9, 14), (4, 7, 7), (6, 12, 12), (6, 13, 11)],
+                         ids=["f43_w16", "f43_w14", "f43_w7", "f63_w12", "f63_w11"])
+def test_fp16_output(m, H, W):
+    """y written as fp16 by every store variant equals the fp32 result rounded once, with and
+    without an epilogue, through the device and the host-buffer entry points, and in the
+    fully quantized mode."""
+    import torch
+    from paper_2412_19867_b200 import binding as b
+    from tests import gpu_util as gu
+    L = Layer(2, 64, 40, H, W, m, 32, "f16", "silu_outlier", "kaiming_chan", 9, 4, 60 + W)
+    conv, (x, w, sB, sG) = gu.make_conv(L)
+    xd = torch.from_numpy(x).to("cuda:0")
+    bias = torch.linspace(-1.0, 1.0, L.K, dtype=torch.float32, device="cuda:0")
+    for epi in (False, True):
+        for fq_mode in ((0, b.WFQ_Y_FP32), (1, b.WFQ_Y_TILE)):
+            conv.set_epilogue(bias if epi else None, b.WFQ_ACT_SILU if epi else b.WFQ_ACT_NONE)
+            b.wfq_plan_set_full_quant(conv.plan, *fq_mode)
+            conv.set_output_dtype("f32")
+            y32 = conv.forward(xd)
+            conv.set_output_dtype("f16")
+            y16 = conv.forward(xd)
+            conv.check_status()
+            assert y16.dtype == torch.float16
+            assert torch.equal(y16, y32.to(torch.float16)), (epi, fq_mode)
+            xh = torch.from_numpy(x).pin_memory()
+            yh = torch.empty(y16.shape, dtype=torch.float16).pin_memory()
+            conv.forward_host(xh, yh)
+            assert torch.equal(yh, y16.cpu())
+    conv.close()
+
+
 def test_host_buffer_entry_point_matches_device_one():
     import torch
     from tests.gpu_util import make_conv
