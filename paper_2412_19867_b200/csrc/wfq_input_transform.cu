@@ -316,6 +316,11 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
     // The contraction kernel launched behind this one may start its prologue and its filter
     // stream now (it waits for this grid's completion before it touches Xq or sX).
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // This kernel itself is launched with programmatic stream serialization: it may become
+    // resident while the kernel before it in the stream (normally the previous layer's output
+    // transform) drains, and waits here, before its first global access, until that kernel has
+    // completed and its writes are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // two strip buffers (the next item is staged while this one is transformed), then Z
     float *Zs = reinterpret_cast<float *>(smem_raw + (1 + prm.dbuf) * prm.strip_bytes);   // [tile][position][CBP]
     const int CBP = prm.CB + 4;   // 16-byte aligned rows an odd number of 16-byte units apart
@@ -460,9 +465,18 @@ template <int M, typename Tin, int GSR, int SPLIT>
 cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stream)
 {
     const K1Params &prm = plan.k1;
-    input_transform_kernel<M, Tin, GSR, SPLIT><<<prm.grid, K1_THREADS, prm.smem, stream>>>(
-        static_cast<const Tin *>(x_dev), plan.ws.Xq, plan.ws.sX, plan.geo, plan.tables, prm);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)prm.grid);
+    cfg.blockDim = dim3(K1_THREADS);
+    cfg.dynamicSmemBytes = prm.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, input_transform_kernel<M, Tin, GSR, SPLIT>, static_cast<const Tin *>(x_dev),
+                              plan.ws.Xq, plan.ws.sX, plan.geo, plan.tables, prm);
 }
 
 // What to do with the instantiation that serves (m, dtype, group size).
