@@ -90,9 +90,14 @@ typedef enum {
                                        2: the tensor-core kernel wherever it applies (fp16 input,
                                        groups of 32 or 64, C a multiple of 64, 16-byte aligned x,
                                        a shape its TMA or bulk staging can describe) */
-    WFQ_DEBUG_SKIP_GEMM_STAGE = 3   /* operand stage (counted from 0) whose loads the first
+    WFQ_DEBUG_SKIP_GEMM_STAGE = 3,  /* operand stage (counted from 0) whose loads the first
                                        CTA of the contraction kernel does not issue (-1 =
                                        none); same purpose as WFQ_DEBUG_SKIP_INPUT_ITEM */
+    WFQ_DEBUG_GEMM_SHAPE = 4        /* 0: the library chooses the contraction's orientation and
+                                       column block; else 100 * orientation (1: accumulator rows are
+                                       tiles, 2: rows are output channels) + columns per unit (16 or
+                                       64 for orientation 1; 16, 32, 48 or 64 for orientation 2).
+                                       Results do not depend on it; for timing experiments */
 } wfq_debug_option_t;
 
 /*

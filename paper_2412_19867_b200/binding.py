@@ -20,6 +20,7 @@ WFQ_Y_FP32, WFQ_Y_TILE, WFQ_Y_ROW = 0, 1, 2
 WFQ_BUF_XQ, WFQ_BUF_SX, WFQ_BUF_WQ, WFQ_BUF_SW, WFQ_BUF_Y, WFQ_BUF_STATUS = range(6)
 WFQ_DEBUG_WAIT_CYCLES, WFQ_DEBUG_SKIP_INPUT_ITEM, WFQ_DEBUG_INPUT_TRANSFORM_KERNEL = range(3)
 WFQ_DEBUG_SKIP_GEMM_STAGE = 3
+WFQ_DEBUG_GEMM_SHAPE = 4
 
 # every symbol include/wfq.h declares
 EXPORTS = [

@@ -514,6 +514,33 @@ wfq_status_t wfq_plan_set_debug_option(wfq_plan_t *plan, wfq_debug_option_t opti
             if (value < -1 || value > 0x7fffffff) return WFQ_ERR_INVALID_ARG;
             plan->debug_skip_gemm_stage = (int)value;
             break;
+        case WFQ_DEBUG_GEMM_SHAPE: {
+            // 0: the library's choice; else 100 * orientation (1 rows = tiles, 2 rows = output
+            // channels) + columns per unit (rows = tiles: 16 or 64; rows = channels: 16, 32, 48, 64)
+            bool swap;
+            int bn;
+            if (value == 0) {
+                wfq::gemm_choose(plan->geo, &swap, &bn);
+            } else {
+                const int orient = (int)(value / 100);
+                bn = (int)(value % 100);
+                if (orient == 1 && (bn == 16 || bn == 64)) swap = false;
+                else if (orient == 2 && (bn == 16 || bn == 32 || bn == 48 || bn == 64)) swap = true;
+                else return WFQ_ERR_INVALID_ARG;
+            }
+            plan->gemm_swap = swap;
+            plan->gemm_bn = bn;
+            const wfq::Geometry &g = plan->geo;
+            if (plan->has_workspace)
+                plan->tmap_xq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_xq, plan->ws.Xq, g.C, g.T, g.P,
+                                                           swap ? bn : wfq::gemm_block_m());
+            if (plan->Wq)
+                plan->tmap_wq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_wq, plan->Wq, g.C, g.K, g.P,
+                                                           swap ? wfq::gemm_block_m() : bn);
+            if ((plan->has_workspace && !plan->tmap_xq_ok) || (plan->Wq && !plan->tmap_wq_ok)) return WFQ_ERR_CUDA;
+            plan->host_chunks = 0;      // the sub-plans of the host-buffer path copy the shape when rebuilt
+            break;
+        }
         default:
             return WFQ_ERR_INVALID_ARG;
     }

@@ -622,7 +622,11 @@ cudaError_t setup_variant()
 // One-time attribute setting for the kernels of this file (per device).
 cudaError_t setup_gemm()
 {
-    cudaError_t e = setup_variant<32, true, true>();
+    cudaError_t e = setup_variant<16, true, true>();
+    if (e == cudaSuccess) e = setup_variant<16, true, false>();
+    if (e == cudaSuccess) e = setup_variant<16, false, true>();
+    if (e == cudaSuccess) e = setup_variant<16, false, false>();
+    if (e == cudaSuccess) e = setup_variant<32, true, true>();
     if (e == cudaSuccess) e = setup_variant<32, true, false>();
     if (e == cudaSuccess) e = setup_variant<48, true, true>();
     if (e == cudaSuccess) e = setup_variant<48, true, false>();
@@ -665,6 +669,15 @@ void gemm_choose(const Geometry &g, bool *swap, int *bn)
 cudaError_t launch_gemm(const wfq_plan &plan, int32_t *acc_dump, cudaStream_t stream, bool pdl)
 {
     const bool dump = acc_dump != nullptr;
+    // 16 columns: never chosen by gemm_choose, only by the debug option (the shape a contraction
+    // fused with the output transform would be confined to by its accumulator space)
+    if (plan.gemm_bn == 16) {
+        if (plan.gemm_swap)
+            return dump ? launch_variant<16, true, true>(plan, acc_dump, stream, pdl)
+                        : launch_variant<16, true, false>(plan, acc_dump, stream, pdl);
+        return dump ? launch_variant<16, false, true>(plan, acc_dump, stream, pdl)
+                    : launch_variant<16, false, false>(plan, acc_dump, stream, pdl);
+    }
     if (plan.gemm_swap) {
         if (plan.gemm_bn == 32)
             return dump ? launch_variant<32, true, true>(plan, acc_dump, stream, pdl)

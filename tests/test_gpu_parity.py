@@ -173,6 +173,36 @@ def test_fp16_output(m, H, W):
     conv.close()
 
 
+@pytest.mark.parametrize("layer", [
+    Layer(2, 128, 96, 24, 24, 4, 64, "f16", "silu_outlier", "kaiming_chan", 9, 5, 1),
+    Layer(1, 192, 200, 12, 12, 6, 32, "f16", "silu_outlier", "kaiming_chan", 9, 5, 2),
+], ids=lambda L: L.name)
+def test_contraction_shapes_agree(layer):
+    """Every orientation / column block the debug option can force gives the library's own
+    result: bit for bit within an orientation (same arithmetic per element), to fp32 rounding
+    across orientations (the two scales are multiplied in the other order)."""
+    import torch
+    from paper_2412_19867_b200 import binding as b
+    from tests import gpu_util as gu
+    _check(layer)
+    conv, (x, w, sB, sG) = gu.make_conv(layer)
+    xd = torch.from_numpy(x).to("cuda:0")
+    ys = {}
+    for shape in (0, 116, 164, 216, 232, 248, 264):
+        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_GEMM_SHAPE, shape)
+        ys[shape] = conv.forward(xd).cpu().numpy()
+        conv.check_status()
+    scale = float(np.max(np.abs(ys[0])))
+    assert np.array_equal(ys[116], ys[164])
+    for shape in (232, 248, 264):
+        assert np.array_equal(ys[216], ys[shape]), shape
+    assert float(np.max(np.abs(ys[116] - ys[216]))) <= 1e-5 * scale
+    assert np.array_equal(ys[0], ys[116]) or np.array_equal(ys[0], ys[216])
+    with pytest.raises(b.WfqError):
+        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_GEMM_SHAPE, 132)
+    conv.close()
+
+
 def test_host_buffer_entry_point_matches_device_one():
     import torch
     from tests.gpu_util import make_conv
