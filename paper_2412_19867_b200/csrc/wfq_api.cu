@@ -507,7 +507,7 @@ wfq_status_t wfq_plan_set_debug_option(wfq_plan_t *plan, wfq_debug_option_t opti
             plan->debug_skip_item = (int)value;
             break;
         case WFQ_DEBUG_INPUT_TRANSFORM_KERNEL:
-            if (value < 0 || value > 2) return WFQ_ERR_INVALID_ARG;
+            if (value < 0 || value > 3) return WFQ_ERR_INVALID_ARG;
             plan->k1_choice = (int)value;
             break;
         case WFQ_DEBUG_SKIP_GEMM_STAGE:

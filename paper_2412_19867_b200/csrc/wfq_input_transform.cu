@@ -33,6 +33,7 @@ namespace {
 
 constexpr int K1_THREADS = 128;
 constexpr int K1_WP = 16;        // staged columns per row (image columns w_base .. w_base+15)
+constexpr int K1_WPV = 24;       // the same where rows are copied in aligned 16-byte pieces (w_base a multiple of 8)
 
 // ---- 1-D input transforms with the standard B^T ------------------------------------
 
@@ -130,6 +131,44 @@ __device__ __forceinline__ void load_patch(const __half *ch, int col0, float (&d
     }
 }
 
+// The same from a strip staged in 16-byte pieces (rows of K1_WPV columns, channel stride a
+// multiple of 16 bytes and an odd number of 16-byte units): 16-byte loads, for which the eight
+// lanes of a quarter warp then hit eight different groups of four banks.  `k0` is the first of
+// the two 16-byte pieces that hold columns col0 .. col0 + NN + 1, WO the 32-bit word of col0
+// inside them (col0 is even); both are the same for all lanes of the warp.
+template <int NN, int WO>
+__device__ __forceinline__ void load_patch_vec(const __half *ch, int k0, float (&d)[NN][NN])
+{
+#pragma unroll
+    for (int a = 0; a < NN; ++a) {
+        const uint4 *row = reinterpret_cast<const uint4 *>(ch + a * K1_WPV) + k0;
+        const uint4 q0 = row[0], q1 = row[1];
+        const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+        float v[NN + 2];
+#pragma unroll
+        for (int i = 0; i < (NN + 2) / 2; ++i) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[WO + i]));
+            v[2 * i] = f.x;
+            v[2 * i + 1] = f.y;
+        }
+#pragma unroll
+        for (int b = 0; b < NN; ++b) d[a][b] = v[b + 1];
+    }
+}
+template <int NN>
+__device__ __forceinline__ void load_patch_vec(const __half *ch, int col0, float (&d)[NN][NN])
+{
+    const int k0 = col0 >> 3;
+    switch ((col0 & 7) >> 1) {            // warp-uniform
+        case 0: load_patch_vec<NN, 0>(ch, k0, d); break;
+        case 1: load_patch_vec<NN, 1>(ch, k0, d); break;
+        case 2: load_patch_vec<NN, 2>(ch, k0, d); break;
+        default: load_patch_vec<NN, 3>(ch, k0, d); break;
+    }
+}
+template <int NN>
+__device__ __forceinline__ void load_patch_vec(const float *, int, float (&)[NN][NN]) {}   // fp16 only
+
 template <int NN>
 __device__ __forceinline__ void load_patch(const float *ch, int col0, float (&d)[NN][NN])
 {
@@ -197,6 +236,11 @@ __device__ __forceinline__ void cp_async_4(uint32_t dst, const void *src, bool v
     const int n = valid ? 4 : 0;   // 0 source bytes: the destination is zero filled
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool valid)
+{
+    const int n = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit()
 {
     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -219,7 +263,30 @@ __device__ __forceinline__ void stage_strip(Tin *sm, const Tin *__restrict__ x, 
     const Tin *ximg = x + ((size_t)img * g.C + c_base) * HW;
     // Each thread owns one (row, column) slot of the strip and walks over the channels,
     // so its bounds test and addresses are computed once.
-    if (sizeof(Tin) == 4 || prm.pair) {
+    if (sizeof(Tin) == 2 && prm.vec16) {
+        // 16-byte pieces: W and w_base are multiples of 8 and x is 16-byte aligned, so a piece
+        // lies inside the image or outside it as a whole
+        constexpr int CPR = K1_WPV / 8;                        // copies per row
+        constexpr int ROWS = K1_THREADS / CPR;
+        constexpr int CSLOTS = ROWS / NN;
+        const int jc = threadIdx.x % CPR;
+        const int rs = threadIdx.x / CPR;
+        const int a = rs % NN, cslot = rs / NN;
+        if (cslot < CSLOTS) {
+            const int h = h_base + a, w = w_base + 8 * jc;
+            const bool ok = h >= 0 && h < g.H && w >= 0 && w < g.W;
+            const Tin *src = ok ? ximg + (size_t)cslot * HW + (size_t)h * g.W + w : x;
+            const size_t src_step = ok ? (size_t)CSLOTS * HW : 0;
+            uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(sm)) +
+                           (uint32_t)((cslot * prm.CS + a * K1_WPV + 8 * jc) * sizeof(Tin));
+            const uint32_t dst_step = (uint32_t)(CSLOTS * prm.CS * sizeof(Tin));
+            for (int c = cslot; c < prm.CB; c += CSLOTS) {
+                cp_async_16(dst, src, ok);
+                src += src_step;
+                dst += dst_step;
+            }
+        }
+    } else if (sizeof(Tin) == 4 || prm.pair) {
         constexpr int EPC = sizeof(Tin) == 4 ? 1 : 2;          // elements per 4-byte copy
         constexpr int CPR = K1_WP / EPC;                       // copies per row
         constexpr int ROWS = K1_THREADS / CPR;                 // rows covered by one pass
@@ -337,8 +404,12 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
         const int cblk = item % prm.NCB, rest = item / prm.NCB;
         const int srow = rest / prm.NCH, chunk = rest - srow * prm.NCH;
         const int img = srow / g.TH, th = srow - img * g.TH;
+        // first staged column: two left of the first tile's first output column, or (16-byte
+        // pieces) the multiple of 8 at or below the first input column
+        const int first = chunk * prm.TB * M - 1;
+        const int w_base = prm.vec16 ? ((first + 8) & ~7) - 8 : first - 1;
         stage_strip<Tin, NN>(reinterpret_cast<Tin *>(smem_raw + buf * prm.strip_bytes), x, g, prm, img,
-                             cblk * prm.CB, th * M - 1, chunk * prm.TB * M - 2);
+                             cblk * prm.CB, th * M - 1, w_base);
         cp_async_commit();
     };
 
@@ -366,11 +437,13 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
         const int c_base = cblk * prm.CB;
 
         // ---- phase 1: transform, one (tile, channel) per thread ----------------------
+        const int voff = tw0 * M - 2 - (((tw0 * M - 1 + 8) & ~7) - 8);   // 16-byte pieces: column of tile 0 minus one
         for (int wt = warp; wt < ntile * cb32; wt += NWARP) {
             const int tl = wt / cb32;
             const int c = (wt - tl * cb32) * 32 + lane;
             float d[NN][NN];
-            load_patch<NN>(strip + c * prm.CS, tl * M, d);
+            if (sizeof(Tin) == 2 && prm.vec16) load_patch_vec<NN>(strip + c * prm.CS, tl * M + voff, d);
+            else load_patch<NN>(strip + c * prm.CS, tl * M, d);
             transform_patch<NN>(d, Zs + (size_t)tl * P * CBP + c, CBP);
         }
         __syncthreads();
@@ -464,7 +537,9 @@ cudaError_t k1_setup()
 template <int M, typename Tin, int GSR, int SPLIT>
 cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stream)
 {
-    const K1Params &prm = plan.k1;
+    // 16-byte pieces need a 16-byte aligned x; the plan holds a second parameter set without them
+    const bool vec = plan.k1v.vec16 && plan.k1_choice != 3 && (reinterpret_cast<uintptr_t>(x_dev) & 15u) == 0;
+    const K1Params &prm = vec ? plan.k1v : plan.k1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)prm.grid);
     cfg.blockDim = dim3(K1_THREADS);
@@ -509,21 +584,23 @@ long long k1_op(K1Op op, int m, bool f16, int gs, const wfq_plan *plan, const vo
 
 }  // namespace
 
-// Work-item shape, shared-memory layout and grid of the cp.async kernel for this plan.
-void plan_input_transform(wfq_plan &plan)
+namespace {
+
+void plan_k1(wfq_plan &plan, K1Params &prm, bool vec16)
 {
     const Geometry &g = plan.geo;
     const bool f16 = plan.in_dtype == WFQ_F16;
     const int NN = g.n, P = g.P, M = g.m;
     const int esz = f16 ? 2 : 4;
-    K1Params &prm = plan.k1;
+    prm.vec16 = vec16 ? 1 : 0;
     prm.TB = (K1_WP - 3) / M;                      // 2 tiles for F(6,3), 3 for F(4,3)
     prm.CB = g.gs;
     if (g.gs == 32 && g.C % 64 == 0) prm.CB = 64;  // two groups per CTA
     // channel stride: an odd number of 32-bit words, so lanes that walk over channels
-    // hit different banks
+    // hit different banks; with 16-byte pieces an odd number of 16-byte units (16-byte loads)
     int cs = NN * K1_WP;
-    if (esz == 2) { cs += 2; if ((cs / 2) % 2 == 0) cs += 2; }
+    if (vec16) { cs = NN * K1_WPV; if ((cs / 8) % 2 == 0) cs += 8; }
+    else if (esz == 2) { cs += 2; if ((cs / 2) % 2 == 0) cs += 2; }
     else if (cs % 2 == 0) cs += 1;
     prm.CS = cs;
     prm.strip_bytes = (prm.CB * cs * esz + 15) / 16 * 16;
@@ -551,6 +628,18 @@ void plan_input_transform(wfq_plan &plan)
     const int per_sm = (int)k1_op(kK1Resident, M, f16, g.gs, nullptr, nullptr, nullptr, (size_t)prm.smem);
     const int resident = per_sm * (plan.sm_count > 0 ? plan.sm_count : 1);
     prm.grid = prm.items < resident ? prm.items : resident;
+}
+
+}  // namespace
+
+// Work-item shape, shared-memory layout and grid of the cp.async kernel for this plan: one set
+// with 4-byte (or 2-byte) copies for any x, and where fp16 rows are whole 16-byte pieces (W a
+// multiple of 8) a second one with 16-byte copies, used when x is 16-byte aligned.
+void plan_input_transform(wfq_plan &plan)
+{
+    plan_k1(plan, plan.k1, false);
+    plan.k1v = plan.k1;
+    if (plan.in_dtype == WFQ_F16 && plan.geo.W % 8 == 0) plan_k1(plan, plan.k1v, true);
 }
 
 cudaError_t setup_input_transform()

@@ -71,6 +71,7 @@ struct K1Params {
     int CS;            // shared-memory channel stride of the strip (elements)
     int strip_bytes;   // bytes of the strip, rounded up to 16
     int pair;          // 1: rows can be copied as aligned element pairs
+    int vec16;         // 1: rows are copied as aligned 16-byte pieces (fp16, W a multiple of 8, x 16-byte aligned)
     int dbuf;          // 1: two strip buffers, the next item is staged during this one
     int smem, grid;    // dynamic shared memory and CTAs of the launch
 };
@@ -119,7 +120,8 @@ struct wfq_plan {
     wfq::ScaleTables tables;
 
     // launch parameters derived from the geometry, the dtype and the device (plan_launches)
-    wfq::K1Params k1;
+    wfq::K1Params k1;          // 4-byte (or 2-byte) copies: any x
+    wfq::K1Params k1v;         // 16-byte copies where the layer allows them (vec16 set), else a copy of k1
     wfq::K1TcPlan k1tc;
     CUtensorMap tmap_x;        // the input tensor as the tensor-core input transform stages it
     const void *tmap_x_base = nullptr;   // x pointer tmap_x was encoded for
@@ -129,7 +131,8 @@ struct wfq_plan {
     bool fq_input = false;     // input transform on integer codes (Eq. quant-B)
     int fq_output = 0;         // output transform: 0 fp32, 1 integer with one scale of Y per tile, 2 per row / column
     wfq::FullQuantTables fq;   // valid once the filters are prepared
-    int k1_choice = 0;         // input-transform kernel: 0 automatic, 1 cp.async, 2 tensor cores where they apply
+    int k1_choice = 0;         // input-transform kernel: 0 automatic, 1 cp.async, 2 tensor cores where they apply,
+                               // 3 cp.async without 16-byte copies
 
     CUtensorMap tmap_xq;       // Xq as (C, T, P) bytes, 128B-swizzled boxes
     CUtensorMap tmap_wq;       // Wq as (C, K, P)

@@ -235,20 +235,26 @@ def test_host_buffer_entry_point_in_chunks_matches_device_one():
     conv.close()
 
 
-def test_input_transform_kernels_agree():
-    """The tensor-core input transform and the cp.async one (selected by a debug option)
-    against the oracle and against each other on the same layer, and a misaligned x
-    (which the tensor-core kernel's TMA descriptor cannot take) falls back by itself."""
+@pytest.mark.parametrize("layer", [
+    Layer(2, 128, 32, 24, 24, 6, 64, "f16", "silu_outlier", "kaiming_chan", 5, 6, 2),
+    Layer(2, 64, 32, 20, 40, 4, 32, "f16", "silu_outlier", "kaiming_chan", 5, 6, 3),
+    Layer(1, 256, 32, 18, 16, 6, 128, "f16", "silu_outlier", "kaiming_chan", 5, 6, 4),
+], ids=lambda L: L.name)
+def test_input_transform_kernels_agree(layer):
+    """The tensor-core input transform, the cp.async one with 16-byte copies (what an aligned
+    fp16 x with W a multiple of 8 gets) and the one with 4-byte copies (debug option, or a
+    misaligned x, which neither a TMA descriptor nor a 16-byte copy can take) against the
+    oracle and against each other on the same layer."""
     import torch
     from oracle import oracle as orc
     from paper_2412_19867_b200 import binding as b
     from tests.gpu_util import make_conv, codes_close, scales_close
-    L = Layer(2, 128, 32, 24, 24, 6, 64, "f16", "silu_outlier", "kaiming_chan", 5, 6, 2)
+    L = layer
     conv, (x, w, sB, sG) = make_conv(L)
     ref = orc.wfq(x, w[:1], L.m, L.gs, sB=sB, sG=sG)
     xbuf = torch.zeros(x.size + 8, dtype=torch.float16, device="cuda")
     got = []
-    for force, offset in ((2, 0), (1, 0), (2, 2)):          # offset in elements: 4-byte aligned only
+    for force, offset in ((2, 0), (1, 0), (2, 2), (3, 0), (0, 0)):          # offset in elements: 4-byte aligned only
         xd = xbuf[offset:offset + x.size].view(x.shape)
         xd.copy_(torch.from_numpy(x))
         b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, force)
@@ -261,7 +267,8 @@ def test_input_transform_kernels_agree():
         scales_close(conv.buffer(b.WFQ_BUF_SX).cpu().numpy()[:, :, :conv.T], ref.sX.transpose(0, 2, 1))
         got.append(xq)
     assert np.mean(got[0] != got[1]) <= 1e-4
-    assert np.array_equal(got[1], got[2])                   # both from the cp.async kernel
+    for other in got[2:]:
+        assert np.array_equal(got[1], other)                # all from the cp.async kernel, either copy width
     conv.close()
 
 
