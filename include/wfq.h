@@ -254,6 +254,18 @@ wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev,
 wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *y_host,
                                    void *stream);
 
+/*
+ * The same without the final wait: the copies and kernels are enqueued and the call returns;
+ * y_host holds the result once `stream` has been waited for (all internal work is joined to
+ * `stream`).  x_host and y_host must stay valid, and x_host unmodified, until then; pageable
+ * host memory makes the copies synchronous with respect to the host.  The plan's staging
+ * buffers are reused by the next call on the same plan, which is ordered after this one when it
+ * uses the same stream; calls on different plans may use different streams so that the copy in
+ * of one layer overlaps the copy out of another.
+ */
+wfq_status_t wfq_conv_forward_host_async(wfq_plan_t *plan, const void *x_host, float *y_host,
+                                         void *stream);
+
 /* The three stages of wfq_conv_forward, separately (tests and profiling). */
 /* Stage 1 (X = S_B V_B x V_B^T S_B, then Q): x_dev -> workspace Xq, sX. */
 wfq_status_t wfq_input_transform_quantize(wfq_plan_t *plan, const void *x_dev, void *stream);

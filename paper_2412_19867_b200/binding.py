@@ -31,6 +31,7 @@ EXPORTS = [
     "wfq_check_device_status", "wfq_plan_destroy", "wfq_status_string", "wfq_version",
     "wfq_quantize_filters_static", "wfq_plan_set_debug_option", "wfq_debug_int8_mma_rate",
     "wfq_plan_set_epilogue", "wfq_plan_set_full_quant", "wfq_plan_set_output_dtype",
+    "wfq_conv_forward_host_async",
 ]
 
 _lib = None
@@ -60,6 +61,7 @@ def load():
     lib.wfq_prepare_filters.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.wfq_conv_forward.argtypes = [vp, vp, vp, vp]
     lib.wfq_conv_forward_host.argtypes = [vp, vp, vp, vp]
+    lib.wfq_conv_forward_host_async.argtypes = [vp, vp, vp, vp]
     lib.wfq_input_transform_quantize.argtypes = [vp, vp, vp]
     lib.wfq_gemm_dequantize.argtypes = [vp, vp]
     lib.wfq_output_transform.argtypes = [vp, vp, vp]
@@ -146,6 +148,10 @@ def wfq_conv_forward(plan, x_dev, y_dev, stream=0):
 
 def wfq_conv_forward_host(plan, x_host, y_host, stream=0):
     _check(load().wfq_conv_forward_host(plan, x_host, y_host, stream), "wfq_conv_forward_host")
+
+
+def wfq_conv_forward_host_async(plan, x_host, y_host, stream=0):
+    _check(load().wfq_conv_forward_host_async(plan, x_host, y_host, stream), "wfq_conv_forward_host_async")
 
 
 def wfq_input_transform_quantize(plan, x_dev, stream=0):
@@ -274,6 +280,14 @@ class Conv:
         """x_host / y_host: CPU tensors (pinned for speed); synchronous."""
         with self.torch.cuda.device(self.device):
             wfq_conv_forward_host(self.plan, x_host.data_ptr(), y_host.data_ptr(), self._stream())
+        return y_host
+
+    def forward_host_async(self, x_host, y_host, stream=None):
+        """The same without the final wait; `stream`: a torch.cuda.Stream (default: the current
+        one).  y_host is valid after that stream has been synchronised."""
+        sptr = self._stream() if stream is None else stream.cuda_stream
+        with self.torch.cuda.device(self.device):
+            wfq_conv_forward_host_async(self.plan, x_host.data_ptr(), y_host.data_ptr(), sptr)
         return y_host
 
     def buffer(self, which):

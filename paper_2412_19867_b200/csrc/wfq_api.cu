@@ -428,8 +428,7 @@ static wfq_status_t setup_host_pipeline(wfq_plan *plan)
     return WFQ_OK;
 }
 
-wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *y_host,
-                                   void *stream)
+static wfq_status_t forward_host(wfq_plan_t *plan, const void *x_host, float *y_host, void *stream, bool wait)
 {
     wfq_status_t s = ready_to_run(plan);
     if (s != WFQ_OK) return s;
@@ -481,7 +480,8 @@ wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *
                 if (err == WFQ_OK) err = WFQ_ERR_CUDA;
             }
         }
-        const cudaError_t se = cudaStreamSynchronize(st);
+        // an error leaves copies queued that must not outlive the call: wait for them either way
+        const cudaError_t se = (wait || err != WFQ_OK) ? cudaStreamSynchronize(st) : cudaSuccess;
         return err != WFQ_OK ? err : cuda_status(se);
     }
 
@@ -491,7 +491,17 @@ wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *
     if (s != WFQ_OK) return s;
     if ((e = cudaMemcpyAsync(y_host, plan->y_stage, yb, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
         return WFQ_ERR_CUDA;
-    return cuda_status(cudaStreamSynchronize(st));
+    return wait ? cuda_status(cudaStreamSynchronize(st)) : WFQ_OK;
+}
+
+wfq_status_t wfq_conv_forward_host(wfq_plan_t *plan, const void *x_host, float *y_host, void *stream)
+{
+    return forward_host(plan, x_host, y_host, stream, true);
+}
+
+wfq_status_t wfq_conv_forward_host_async(wfq_plan_t *plan, const void *x_host, float *y_host, void *stream)
+{
+    return forward_host(plan, x_host, y_host, stream, false);
 }
 
 wfq_status_t wfq_plan_set_debug_option(wfq_plan_t *plan, wfq_debug_option_t option, long long value)

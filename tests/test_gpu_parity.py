@@ -203,6 +203,36 @@ def test_contraction_shapes_agree(layer):
     conv.close()
 
 
+def test_asynchronous_host_buffer_entry_point():
+    """Two layers through wfq_conv_forward_host_async on two streams, repeatedly, against the
+    synchronous entry point (one of them large enough for the chunked path)."""
+    import torch
+    from tests import gpu_util as gu
+    layers = [Layer(4, 64, 192, 64, 64, 4, 32, "f16", "silu_outlier", "kaiming_chan", 9, 6, 1),
+              Layer(1, 64, 32, 13, 11, 6, 64, "f16", "silu_outlier", "kaiming_chan", 9, 6, 2)]
+    convs, xs, want, got = [], [], [], []
+    for L in layers:
+        conv, (x, w, sB, sG) = gu.make_conv(L)
+        xh = torch.from_numpy(x).pin_memory()
+        yh = torch.empty((L.N, L.K, L.H, L.W), dtype=torch.float32).pin_memory()
+        conv.forward_host(xh, yh)
+        convs.append(conv); xs.append(xh); want.append(yh.clone())
+        got.append(torch.full(yh.shape, float("nan"), dtype=torch.float32).pin_memory())
+    streams = [torch.cuda.Stream("cuda:0") for _ in layers]
+    for rep in range(3):
+        for conv, xh, yh, st in zip(convs, xs, got, streams):
+            conv.forward_host_async(xh, yh, st)
+        for st in streams:
+            st.synchronize()
+        for a, b_ in zip(want, got):
+            assert torch.equal(a, b_)
+        for yh in got:
+            yh.fill_(float("nan"))
+    for conv in convs:
+        conv.check_status()
+        conv.close()
+
+
 def test_host_buffer_entry_point_matches_device_one():
     import torch
     from tests.gpu_util import make_conv
