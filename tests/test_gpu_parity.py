@@ -1,7 +1,7 @@
 """GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle
 on the same seeded tensors.
 
-Bars (from the build's statement of the task):
+Bars:
   * int32 group accumulators: bit exact given identical int8 operands;
   * int8 Winograd-domain tensors: bit exact except at most 1e-4 of the elements, off
     by one LSB (fp32 transform on the GPU vs fp64-then-round in the oracle);
