@@ -242,6 +242,23 @@ wfq_status_t wfq_quantize_filters_static(const float *w_dev, int K, int C, int m
 wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev, void *stream);
 
 /*
+ * Prepared filters as a host blob, so that wfq_prepare_filters can run once, offline, and a later
+ * process only loads its result (the filter path is offline in the paper as well, Section 4.1).
+ * The blob holds a 256-byte header (layer shape, tile and group size, the three scale vectors in
+ * fp64), Wq [P][K][C] int8 and sW [P][G][Kp] fp32; it is tied to those parameters, not to the
+ * batch size or the image size.
+ *   wfq_filters_bytes   size of the blob for this plan
+ *   wfq_filters_export  host_buf (host, >= that size, caller-owned) receives the blob of a
+ *                       prepared plan; synchronous with respect to `stream`
+ *   wfq_filters_import  makes the plan prepared from a blob written for the same C, K, tile and
+ *                       group size (WFQ_ERR_INVALID_ARG otherwise, plan unchanged); the blob is
+ *                       copied before the call returns
+ */
+size_t wfq_filters_bytes(const wfq_plan_t *plan);
+wfq_status_t wfq_filters_export(wfq_plan_t *plan, void *host_buf, size_t bytes, void *stream);
+wfq_status_t wfq_filters_import(wfq_plan_t *plan, const void *host_buf, size_t bytes, void *stream);
+
+/*
  * Same computation with HOST buffers: copies x to the device, runs the three kernels,
  * copies y back, then waits for `stream` (synchronous).  The plan allocates device
  * staging for x and y on first use.  x_host/y_host should be pinned for full copy speed.

@@ -31,7 +31,7 @@ EXPORTS = [
     "wfq_check_device_status", "wfq_plan_destroy", "wfq_status_string", "wfq_version",
     "wfq_quantize_filters_static", "wfq_plan_set_debug_option", "wfq_debug_int8_mma_rate",
     "wfq_plan_set_epilogue", "wfq_plan_set_full_quant", "wfq_plan_set_output_dtype",
-    "wfq_conv_forward_host_async",
+    "wfq_conv_forward_host_async", "wfq_filters_bytes", "wfq_filters_export", "wfq_filters_import",
 ]
 
 _lib = None
@@ -62,6 +62,10 @@ def load():
     lib.wfq_conv_forward.argtypes = [vp, vp, vp, vp]
     lib.wfq_conv_forward_host.argtypes = [vp, vp, vp, vp]
     lib.wfq_conv_forward_host_async.argtypes = [vp, vp, vp, vp]
+    lib.wfq_filters_bytes.argtypes = [vp]
+    lib.wfq_filters_bytes.restype = ctypes.c_size_t
+    lib.wfq_filters_export.argtypes = [vp, vp, ctypes.c_size_t, vp]
+    lib.wfq_filters_import.argtypes = [vp, vp, ctypes.c_size_t, vp]
     lib.wfq_input_transform_quantize.argtypes = [vp, vp, vp]
     lib.wfq_gemm_dequantize.argtypes = [vp, vp]
     lib.wfq_output_transform.argtypes = [vp, vp, vp]
@@ -148,6 +152,24 @@ def wfq_conv_forward(plan, x_dev, y_dev, stream=0):
 
 def wfq_conv_forward_host(plan, x_host, y_host, stream=0):
     _check(load().wfq_conv_forward_host(plan, x_host, y_host, stream), "wfq_conv_forward_host")
+
+
+def wfq_filters_bytes(plan):
+    return int(load().wfq_filters_bytes(plan))
+
+
+def wfq_filters_export(plan, stream=0):
+    """The prepared filters of the plan as a bytes-like host buffer (ctypes array)."""
+    n = wfq_filters_bytes(plan)
+    buf = (ctypes.c_char * n)()
+    _check(load().wfq_filters_export(plan, ctypes.cast(buf, ctypes.c_void_p), n, stream), "wfq_filters_export")
+    return buf
+
+
+def wfq_filters_import(plan, blob, stream=0):
+    raw = bytes(blob)
+    _check(load().wfq_filters_import(plan, ctypes.cast(ctypes.c_char_p(raw), ctypes.c_void_p), len(raw), stream),
+           "wfq_filters_import")
 
 
 def wfq_conv_forward_host_async(plan, x_host, y_host, stream=0):

@@ -248,6 +248,54 @@ wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t byte
     return WFQ_OK;
 }
 
+// The per-position products of the plan's scale vectors (rounded once from fp64).
+static void fill_scale_tables(wfq_plan *plan)
+{
+    const wfq::Geometry &g = plan->geo;
+    const double *stdB = g.m == 4 ? kStdSB4 : kStdSB6;
+    for (int i = 0; i < g.n; ++i)
+        for (int j = 0; j < g.n; ++j) {
+            const double f = (plan->sB[i] / stdB[i]) * (plan->sB[j] / stdB[j]);
+            plan->tables.in_scale[i * g.n + j] = (float)f;
+            plan->tables.in_scale_lo[i * g.n + j] = (float)(f - (double)(float)f);
+            plan->tables.out_scale[i * g.n + j] = (float)(plan->sA[i] * plan->sA[j]);
+        }
+}
+
+// Device buffers of the prepared filters and the status word (allocated once per plan).
+static wfq_status_t ensure_filter_buffers(wfq_plan *plan, cudaStream_t stream)
+{
+    const wfq::Geometry &g = plan->geo;
+    wfq_status_t bs = bind_device(plan);
+    if (bs != WFQ_OK) return bs;
+    cudaError_t e;
+    const size_t wq_bytes = (size_t)g.P * g.K * g.C;
+    const size_t sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
+    if (!plan->Wq && (e = cudaMalloc(&plan->Wq, wq_bytes)) != cudaSuccess) return cuda_status(e);
+    if (!plan->sW) {
+        if ((e = cudaMalloc(&plan->sW, sw_bytes)) != cudaSuccess) return cuda_status(e);
+        // the padding columns k >= K stay zero
+        if ((e = cudaMemsetAsync(plan->sW, 0, sw_bytes, stream)) != cudaSuccess) return WFQ_ERR_CUDA;
+    }
+    if (!plan->status) {
+        if ((e = cudaMalloc(&plan->status, 4 * sizeof(int))) != cudaSuccess) return cuda_status(e);
+        if ((e = cudaMemsetAsync(plan->status, 0, 4 * sizeof(int), stream)) != cudaSuccess) return WFQ_ERR_CUDA;
+    }
+    return WFQ_OK;
+}
+
+// What follows once Wq and sW are in place.
+static wfq_status_t finish_filters(wfq_plan *plan)
+{
+    const wfq::Geometry &g = plan->geo;
+    plan->tmap_wq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_wq, plan->Wq, g.C, g.K, g.P,
+                                               plan->gemm_swap ? wfq::gemm_block_m() : plan->gemm_bn);
+    if (!plan->tmap_wq_ok) return WFQ_ERR_CUDA;
+    wfq::build_full_quant_tables(*plan);
+    plan->prepared = true;
+    return WFQ_OK;
+}
+
 wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const float *sB_host,
                                  const float *sG_host, const float *sA_host, void *stream)
 {
@@ -269,32 +317,12 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
         }
         plan->sB[i] = b; plan->sG[i] = s; plan->sA[i] = a;
     }
-    for (int i = 0; i < g.n; ++i)
-        for (int j = 0; j < g.n; ++j) {
-            const double f = (plan->sB[i] / stdB[i]) * (plan->sB[j] / stdB[j]);
-            plan->tables.in_scale[i * g.n + j] = (float)f;
-            plan->tables.in_scale_lo[i * g.n + j] = (float)(f - (double)(float)f);
-            plan->tables.out_scale[i * g.n + j] = (float)(plan->sA[i] * plan->sA[j]);
-        }
+    fill_scale_tables(plan);
 
-    wfq_status_t bs = bind_device(plan);
+    wfq_status_t bs = ensure_filter_buffers(plan, as_stream(stream));
     if (bs != WFQ_OK) return bs;
     cudaError_t e;
-
     const size_t wq_bytes = (size_t)g.P * g.K * g.C;
-    const size_t sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
-    if (!plan->Wq && (e = cudaMalloc(&plan->Wq, wq_bytes)) != cudaSuccess) return cuda_status(e);
-    if (!plan->sW) {
-        if ((e = cudaMalloc(&plan->sW, sw_bytes)) != cudaSuccess) return cuda_status(e);
-        // the padding columns k >= K stay zero
-        if ((e = cudaMemsetAsync(plan->sW, 0, sw_bytes, as_stream(stream))) != cudaSuccess)
-            return WFQ_ERR_CUDA;
-    }
-    if (!plan->status) {
-        if ((e = cudaMalloc(&plan->status, 4 * sizeof(int))) != cudaSuccess) return cuda_status(e);
-        if ((e = cudaMemsetAsync(plan->status, 0, 4 * sizeof(int), as_stream(stream))) != cudaSuccess)
-            return WFQ_ERR_CUDA;
-    }
     // fp32 transformed filters between the two kernels: stream-ordered allocation, released
     // in stream order after the quantization kernel, so the call neither blocks nor holds
     // the temporary (four times the size of Wq) any longer than the kernels need it
@@ -304,13 +332,75 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
     e = wfq::launch_filter_prep(*plan, w_dev, static_cast<float *>(w32), as_stream(stream));
     cudaError_t e2 = cudaFreeAsync(w32, as_stream(stream));
     if (e != cudaSuccess || e2 != cudaSuccess) return WFQ_ERR_CUDA;
+    return finish_filters(plan);
+}
 
-    plan->tmap_wq_ok = wfq::encode_tmap_bytes3d(&plan->tmap_wq, plan->Wq, g.C, g.K, g.P,
-                                               plan->gemm_swap ? wfq::gemm_block_m() : plan->gemm_bn);
-    if (!plan->tmap_wq_ok) return WFQ_ERR_CUDA;
-    wfq::build_full_quant_tables(*plan);
-    plan->prepared = true;
-    return WFQ_OK;
+// ---- prepared filters as a host blob ------------------------------------------------------
+namespace {
+struct FilterBlobHeader {
+    char magic[8];                       // "WFQFILT1"
+    int32_t m, C, K, gs, P, G, Kp, reserved;
+    double sB[wfq::kMaxN], sG[wfq::kMaxN], sA[wfq::kMaxN];
+    char pad[256 - 8 - 8 * 4 - 3 * 8 * wfq::kMaxN];
+};
+static_assert(sizeof(FilterBlobHeader) == 256, "header is 256 bytes");
+const char kBlobMagic[8] = {'W', 'F', 'Q', 'F', 'I', 'L', 'T', '1'};
+}  // namespace
+
+size_t wfq_filters_bytes(const wfq_plan_t *plan)
+{
+    if (!plan) return 0;
+    const wfq::Geometry &g = plan->geo;
+    return sizeof(FilterBlobHeader) + (size_t)g.P * g.K * g.C + (size_t)g.P * g.G * g.Kp * sizeof(float);
+}
+
+wfq_status_t wfq_filters_export(wfq_plan_t *plan, void *host_buf, size_t bytes, void *stream)
+{
+    if (!plan || !host_buf) return WFQ_ERR_INVALID_ARG;
+    if (!plan->prepared) return WFQ_ERR_NOT_PREPARED;
+    if (bytes < wfq_filters_bytes(plan)) return WFQ_ERR_INVALID_ARG;
+    const wfq::Geometry &g = plan->geo;
+    FilterBlobHeader h;
+    memset(&h, 0, sizeof(h));
+    memcpy(h.magic, kBlobMagic, 8);
+    h.m = g.m; h.C = g.C; h.K = g.K; h.gs = g.gs; h.P = g.P; h.G = g.G; h.Kp = g.Kp;
+    for (int i = 0; i < g.n; ++i) { h.sB[i] = plan->sB[i]; h.sG[i] = plan->sG[i]; h.sA[i] = plan->sA[i]; }
+    memcpy(host_buf, &h, sizeof(h));
+    char *dst = static_cast<char *>(host_buf) + sizeof(h);
+    const size_t wq_bytes = (size_t)g.P * g.K * g.C, sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemcpyAsync(dst, plan->Wq, wq_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(dst + wq_bytes, plan->sW, sw_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return WFQ_ERR_CUDA;
+    return cuda_status(cudaStreamSynchronize(st));
+}
+
+wfq_status_t wfq_filters_import(wfq_plan_t *plan, const void *host_buf, size_t bytes, void *stream)
+{
+    if (!plan || !host_buf || bytes < sizeof(FilterBlobHeader)) return WFQ_ERR_INVALID_ARG;
+    const wfq::Geometry &g = plan->geo;
+    FilterBlobHeader h;
+    memcpy(&h, host_buf, sizeof(h));
+    if (memcmp(h.magic, kBlobMagic, 8) != 0 || h.m != g.m || h.C != g.C || h.K != g.K || h.gs != g.gs ||
+        h.P != g.P || h.G != g.G || h.Kp != g.Kp || bytes < wfq_filters_bytes(plan))
+        return WFQ_ERR_INVALID_ARG;
+    for (int i = 0; i < g.n; ++i)
+        if (!std::isfinite(h.sB[i]) || !std::isfinite(h.sG[i]) || !std::isfinite(h.sA[i]) || h.sB[i] == 0.0 ||
+            h.sG[i] == 0.0 || h.sA[i] == 0.0)
+            return WFQ_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    wfq_status_t bs = ensure_filter_buffers(plan, st);
+    if (bs != WFQ_OK) return bs;
+    for (int i = 0; i < g.n; ++i) { plan->sB[i] = h.sB[i]; plan->sG[i] = h.sG[i]; plan->sA[i] = h.sA[i]; }
+    fill_scale_tables(plan);
+    const char *src = static_cast<const char *>(host_buf) + sizeof(h);
+    const size_t wq_bytes = (size_t)g.P * g.K * g.C, sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
+    if (cudaMemcpyAsync(plan->Wq, src, wq_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(plan->sW, src + wq_bytes, sw_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return WFQ_ERR_CUDA;
+    // the caller may free or change the blob when this returns
+    if (cudaStreamSynchronize(st) != cudaSuccess) return WFQ_ERR_CUDA;
+    return finish_filters(plan);
 }
 
 wfq_status_t wfq_input_transform_quantize(wfq_plan_t *plan, const void *x_dev, void *stream)

@@ -106,6 +106,13 @@ def test_null_plan_is_rejected_everywhere(lib):
     assert lib.wfq_plan_set_workspace(None, fake, 0) == b.WFQ_ERR_INVALID_ARG
     assert lib.wfq_prepare_filters(None, fake, None, None, None, None) == b.WFQ_ERR_INVALID_ARG
     assert lib.wfq_check_device_status(None, None, None) == b.WFQ_ERR_INVALID_ARG
+    assert lib.wfq_conv_forward_host_async(None, fake, fake, None) == b.WFQ_ERR_INVALID_ARG
+    assert lib.wfq_plan_set_epilogue(None, None, 0) == b.WFQ_ERR_INVALID_ARG
+    assert lib.wfq_plan_set_output_dtype(None, 0) == b.WFQ_ERR_INVALID_ARG
+    assert lib.wfq_plan_set_full_quant(None, 0, 0) == b.WFQ_ERR_INVALID_ARG
+    assert lib.wfq_filters_bytes(None) == 0
+    assert lib.wfq_filters_export(None, fake, 0, None) == b.WFQ_ERR_INVALID_ARG
+    assert lib.wfq_filters_import(None, fake, 0, None) == b.WFQ_ERR_INVALID_ARG
 
 
 def test_status_strings(lib):

@@ -203,6 +203,46 @@ def test_contraction_shapes_agree(layer):
     conv.close()
 
 
+def test_filters_export_and_import():
+    """A plan made ready from an exported blob computes what the plan that prepared the filters
+    computes (also for another batch and image size, and in the fully quantized mode); a blob
+    for other parameters or a damaged one is refused and leaves the plan unprepared."""
+    import torch
+    from paper_2412_19867_b200 import binding as b
+    from tests import gpu_util as gu
+    L = Layer(2, 128, 72, 20, 24, 6, 64, "f16", "silu_outlier", "kaiming_chan", 9, 7, 1)
+    conv, (x, w, sB, sG) = gu.make_conv(L)
+    blob = b.wfq_filters_export(conv.plan, conv._stream())
+    assert len(blob) == b.wfq_filters_bytes(conv.plan)
+    xd = torch.from_numpy(x).to("cuda:0")
+    for N, H, W in ((L.N, L.H, L.W), (1, 9, 14)):
+        a = b.Conv(N, L.C, L.K, H, W, L.m, L.gs, L.dtype)
+        a.prepare(torch.from_numpy(w).to("cuda:0"), list(sB), list(sG))
+        c = b.Conv(N, L.C, L.K, H, W, L.m, L.gs, L.dtype)
+        b.wfq_filters_import(c.plan, blob, c._stream())
+        xs = xd[:N, :, :H, :W].contiguous()
+        for mode in ((0, b.WFQ_Y_FP32), (1, b.WFQ_Y_ROW)):
+            b.wfq_plan_set_full_quant(a.plan, *mode)
+            b.wfq_plan_set_full_quant(c.plan, *mode)
+            assert torch.equal(a.forward(xs), c.forward(xs))
+        c.check_status()
+        a.close(); c.close()
+    other = b.Conv(1, L.C, L.K + 8, 8, 8, L.m, L.gs, L.dtype)
+    with pytest.raises(b.WfqError):
+        b.wfq_filters_import(other.plan, blob)
+    bad = bytearray(bytes(blob)); bad[0] ^= 0xff
+    same = b.Conv(1, L.C, L.K, 8, 8, L.m, L.gs, L.dtype)
+    with pytest.raises(b.WfqError):
+        b.wfq_filters_import(same.plan, bytes(bad))
+    with pytest.raises(b.WfqError):
+        b.wfq_filters_import(same.plan, bytes(blob)[:1000])
+    with pytest.raises(b.WfqError):                      # still not prepared
+        same.forward(torch.zeros((1, L.C, 8, 8), dtype=torch.float16, device="cuda:0"))
+    with pytest.raises(b.WfqError):
+        b.wfq_filters_export(same.plan)
+    other.close(); same.close(); conv.close()
+
+
 def test_asynchronous_host_buffer_entry_point():
     """Two layers through wfq_conv_forward_host_async on two streams, repeatedly, against the
     synchronous entry point (one of them large enough for the chunked path)."""
