@@ -701,14 +701,38 @@ def run_wfq(args):
                 conv.forward_host(x, y)          # synchronous: copies + kernels + copy back
         torch.cuda.synchronize(dev)
         dts = max_over_ranks(time.perf_counter() - t0, dev)
+        # the same with y written and copied out as fp16 (wfq_plan_set_output_dtype): half the bytes out
+        for conv in wk.convs:
+            conv.set_output_dtype("f16")
+        yh16 = [torch.empty(y.shape, dtype=torch.float16).pin_memory() for y in wk.ys]
+
+        def e2e_step16():
+            for i, (conv, x, y) in enumerate(zip(wk.convs, xh, yh16)):
+                conv.forward_host_async(x, y, side[i % 3])
+            for st in side:
+                st.synchronize()
+
+        e2e_step16()
+        same16 = all(torch.equal(a.to(torch.float16), b_) for a, b_ in zip(want, yh16))
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(esteps):
+            e2e_step16()
+        torch.cuda.synchronize(dev)
+        dt16 = max_over_ranks(time.perf_counter() - t0, dev)
+        for conv in wk.convs:
+            conv.set_output_dtype("f32")
         e2e = {"value": replica_throughput(wk.step_ops, world, dt * 1e3 / esteps), "unit": UNIT,
                "h2d_bytes_per_step": int(sum(x.numel() * x.element_size() for x in xh)),
                "d2h_bytes_per_step": int(sum(y.numel() * 4 for y in yh)), "steps": esteps,
                "api": "wfq_conv_forward_host_async per layer on three streams, one wait per step",
                "matches_synchronous_result": bool(same),
                "serial": {"value": replica_throughput(wk.step_ops, world, dts * 1e3 / esteps), "unit": UNIT,
-                          "api": "wfq_conv_forward_host per layer"}}
-        del xh, yh, want
+                          "api": "wfq_conv_forward_host per layer"},
+               "fp16_output": {"value": replica_throughput(wk.step_ops, world, dt16 * 1e3 / esteps), "unit": UNIT,
+                               "d2h_bytes_per_step": int(sum(y.numel() * 2 for y in yh16)),
+                               "equals_fp32_result_rounded_once": bool(same16)}}
+        del xh, yh, yh16, want
 
     layers, tensors = wk.layers, wk.tensors
     launch_mode = wk.launch_mode
