@@ -63,6 +63,10 @@ SMALL = [
     Layer(1, 64, 32, 24, 136, 4, 64, "f16", "silu_outlier", "kaiming_chan", 5, 0, 1),   # W = 136: chunks
     Layer(1, 128, 32, 20, 64, 6, 32, "f16", "silu_outlier", "kaiming_chan", 5, 5, 1),   # 11 tiles per row
     Layer(5, 64, 32, 10, 16, 6, 64, "f16", "relu_heavy", "kaiming", 2, 0, 2),           # 3 tiles per row
+    # 16-byte staging of the input transform (fp16, W a multiple of 8) with the other group paths:
+    # groups of 256 (four lanes per group) and of 96 (group read twice from shared memory)
+    Layer(1, 512, 32, 16, 16, 6, 256, "f16", "silu_outlier", "kaiming_chan", 5, 9, 1),
+    Layer(2, 192, 32, 12, 24, 4, 96, "f16", "silu_outlier", "kaiming_chan", 5, 9, 2),
 ]
 
 
