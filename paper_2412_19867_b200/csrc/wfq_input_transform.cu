@@ -419,7 +419,9 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
         const int buf = prm.dbuf ? (it & 1) : 0;
         const int next = item + gridDim.x;
         if (!prm.dbuf) {
-            stage_item(item, 0);               // very large channel blocks: one buffer only
+            // one buffer: this item's copies were issued after the previous item's patches had been
+            // read (below), and landed while that item was quantized
+            if (it == 0) stage_item(item, 0);
             cp_async_wait_group<0>();
         } else if (next < prm.items) {
             stage_item(next, buf ^ 1);
@@ -447,6 +449,7 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
             transform_patch<NN>(d, Zs + (size_t)tl * P * CBP + c, CBP);
         }
         __syncthreads();
+        if (!prm.dbuf && next < prm.items) stage_item(next, 0);   // the strip buffer is free: refill it now
 
         // ---- phase 2: quantize, one (tile, group, position) per thread -------------------
         // X = Z * (caller's per-position factor) is formed here, one rounding, as the
