@@ -30,9 +30,23 @@ namespace {
 constexpr double kQmax = 127.0;
 
 // Q(v / s) for s = amax / 127 > 0: fp64 division, round half to even, clipped.
-__device__ __forceinline__ int code_of(double v, double s)
+__device__ __noinline__ int code_by_division(double v, double s)
 {
     const double q = rint(__ddiv_rn(v, s));
+    return (int)fmin(fmax(q, -kQmax), kQmax);
+}
+// The same code without the division in all but rare cases: a candidate from the reciprocal
+// (rinv = 1 / s, one division per scale instead of one per element), its remainder v - q s by one
+// fused multiply-add, a step to the neighbour if the remainder says so, and the division itself
+// where the remainder is within 1e-9 s of half a step (there the rounding of the quotient
+// decides, and the definition is the division).
+__device__ __forceinline__ int code_of(double v, double s, double rinv)
+{
+    double q = rint(__dmul_rn(v, rinv));
+    const double r = __fma_rn(-q, s, v);
+    const double h = 0.5 * s, ar = fabs(r);
+    if (fabs(ar - h) <= 1e-9 * s) return code_by_division(v, s);
+    if (ar > h) q += r > 0.0 ? 1.0 : -1.0;
     return (int)fmin(fmax(q, -kQmax), kQmax);
 }
 
@@ -89,11 +103,12 @@ __global__ void input_transform_int_kernel(const Tin *__restrict__ x, int8_t *__
 
     // Q(x / s_qx), then the two integer products with the codes of S_B V_B
     const double sqx = __ddiv_rn((double)amax, kQmax);
+    const double rqx = amax > 0.f ? __ddiv_rn(1.0, sqx) : 0.0;
     int q[NN][NN];
 #pragma unroll
     for (int a = 0; a < NN; ++a)
 #pragma unroll
-        for (int b = 0; b < NN; ++b) q[a][b] = amax > 0.f ? code_of((double)d[a][b], sqx) : 0;
+        for (int b = 0; b < NN; ++b) q[a][b] = amax > 0.f ? code_of((double)d[a][b], sqx, rqx) : 0;
     int tmp[NN][NN];
 #pragma unroll
     for (int i = 0; i < NN; ++i)
@@ -161,12 +176,13 @@ output_transform_int_kernel(const float *__restrict__ Y, float *__restrict__ y, 
 #pragma unroll
             for (int j = 0; j < NN; ++j) amax = fmaxf(amax, fabsf(v[i][j]));
         const double sqY = __ddiv_rn((double)amax, kQmax);
+        const double rqY = amax > 0.f ? __ddiv_rn(1.0, sqY) : 0.0;
         int tmp[NN][M];         // Q(Y) Q(S_A V_A^T): [i][v]
 #pragma unroll
         for (int i = 0; i < NN; ++i) {
             int q[NN];
 #pragma unroll
-            for (int j = 0; j < NN; ++j) q[j] = amax > 0.f ? code_of((double)v[i][j], sqY) : 0;
+            for (int j = 0; j < NN; ++j) q[j] = amax > 0.f ? code_of((double)v[i][j], sqY, rqY) : 0;
 #pragma unroll
             for (int c = 0; c < M; ++c) {
                 int s = 0;
@@ -193,9 +209,10 @@ output_transform_int_kernel(const float *__restrict__ Y, float *__restrict__ y, 
 #pragma unroll
             for (int j = 0; j < NN; ++j) amax = fmaxf(amax, fabsf(v[i][j]));
             const double sr = __ddiv_rn((double)amax, kQmax);
+            const double rr = amax > 0.f ? __ddiv_rn(1.0, sr) : 0.0;
             int q[NN];
 #pragma unroll
-            for (int j = 0; j < NN; ++j) q[j] = amax > 0.f ? code_of((double)v[i][j], sr) : 0;
+            for (int j = 0; j < NN; ++j) q[j] = amax > 0.f ? code_of((double)v[i][j], sr, rr) : 0;
 #pragma unroll
             for (int c = 0; c < M; ++c) {
                 int s = 0;
@@ -210,9 +227,10 @@ output_transform_int_kernel(const float *__restrict__ Y, float *__restrict__ y, 
 #pragma unroll
             for (int i = 0; i < NN; ++i) amax = fmax(amax, fabs(Z[i][c]));
             const double sc = __ddiv_rn(amax, kQmax);
+            const double rc = amax > 0.0 ? __ddiv_rn(1.0, sc) : 0.0;
             int q[NN];
 #pragma unroll
-            for (int i = 0; i < NN; ++i) q[i] = amax > 0.0 ? code_of(Z[i][c], sc) : 0;
+            for (int i = 0; i < NN; ++i) q[i] = amax > 0.0 ? code_of(Z[i][c], sc, rc) : 0;
 #pragma unroll
             for (int u = 0; u < M; ++u) {
                 int s = 0;
