@@ -63,6 +63,9 @@ typedef enum {
 
 typedef enum { WFQ_F32 = 0, WFQ_F16 = 1 } wfq_dtype_t;
 
+/* Memory layout of the input x: [N][C][H][W] (default) or [N][H][W][C]. */
+typedef enum { WFQ_NCHW = 0, WFQ_NHWC = 1 } wfq_layout_t;
+
 /* Activation applied by the output transform after the optional bias. */
 typedef enum { WFQ_ACT_NONE = 0, WFQ_ACT_RELU = 1, WFQ_ACT_SILU = 2 } wfq_activation_t;
 
@@ -124,6 +127,16 @@ wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype);
  * Host only; takes effect from the next forward call.  Default: no bias, no activation.
  */
 wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_activation_t act);
+
+/*
+ * Layout of x.  With WFQ_NHWC, `x_dev` / `x_host` of the forward calls hold x[N][H][W][C] (same
+ * element type as set by wfq_plan_set_input_dtype) and x_dev must be 16-byte aligned
+ * (WFQ_ERR_CUDA from the forward call otherwise); the input transform then stages each work
+ * item's strip with one TMA tensor copy (channels innermost) instead of per-thread copies.  The
+ * result is the same bit for bit as for the NCHW tensor with the same values; y stays
+ * [N][K][H][W].  Not available together with the integer input transform.  Host only.
+ */
+wfq_status_t wfq_plan_set_input_layout(wfq_plan_t *plan, wfq_layout_t layout);
 
 /*
  * Element type of the output y: WFQ_F32 (default) or WFQ_F16.  With WFQ_F16 the output transform

@@ -17,6 +17,7 @@ WFQ_STATIC_SCRATCH_FLOATS = 4 * 1024 * 1024
 WFQ_F32, WFQ_F16 = 0, 1
 WFQ_ACT_NONE, WFQ_ACT_RELU, WFQ_ACT_SILU = 0, 1, 2
 WFQ_Y_FP32, WFQ_Y_TILE, WFQ_Y_ROW = 0, 1, 2
+WFQ_NCHW, WFQ_NHWC = 0, 1
 WFQ_BUF_XQ, WFQ_BUF_SX, WFQ_BUF_WQ, WFQ_BUF_SW, WFQ_BUF_Y, WFQ_BUF_STATUS = range(6)
 WFQ_DEBUG_WAIT_CYCLES, WFQ_DEBUG_SKIP_INPUT_ITEM, WFQ_DEBUG_INPUT_TRANSFORM_KERNEL = range(3)
 WFQ_DEBUG_SKIP_GEMM_STAGE = 3
@@ -32,6 +33,7 @@ EXPORTS = [
     "wfq_quantize_filters_static", "wfq_plan_set_debug_option", "wfq_debug_int8_mma_rate",
     "wfq_plan_set_epilogue", "wfq_plan_set_full_quant", "wfq_plan_set_output_dtype",
     "wfq_conv_forward_host_async", "wfq_filters_bytes", "wfq_filters_export", "wfq_filters_import",
+    "wfq_plan_set_input_layout",
 ]
 
 _lib = None
@@ -77,6 +79,7 @@ def load():
     lib.wfq_plan_set_epilogue.argtypes = [vp, vp, ci]
     lib.wfq_plan_set_full_quant.argtypes = [vp, ci, ci]
     lib.wfq_plan_set_output_dtype.argtypes = [vp, ci]
+    lib.wfq_plan_set_input_layout.argtypes = [vp, ci]
     lib.wfq_plan_set_debug_option.argtypes = [vp, ci, ctypes.c_longlong]
     lib.wfq_debug_int8_mma_rate.argtypes = [vp, ci, ci, ctypes.POINTER(ctypes.c_longlong), vp]
     lib.wfq_status_string.argtypes = [ci]
@@ -121,6 +124,10 @@ def wfq_plan_set_input_dtype(plan, dtype):
 
 def wfq_plan_set_epilogue(plan, bias_dev, act=WFQ_ACT_NONE):
     _check(load().wfq_plan_set_epilogue(plan, bias_dev, act), "wfq_plan_set_epilogue")
+
+
+def wfq_plan_set_input_layout(plan, layout):
+    _check(load().wfq_plan_set_input_layout(plan, layout), "wfq_plan_set_input_layout")
 
 
 def wfq_plan_set_output_dtype(plan, dtype):
@@ -272,6 +279,11 @@ class Conv:
         with torch.cuda.device(self.device):
             wfq_prepare_filters(self.plan, w.data_ptr(), sB, sG, sA, self._stream())
 
+    def set_input_layout(self, layout):
+        """"nchw" (default) or "nhwc": forward() then takes x of shape (N, H, W, C)."""
+        self.in_layout = layout
+        wfq_plan_set_input_layout(self.plan, WFQ_NHWC if layout == "nhwc" else WFQ_NCHW)
+
     def set_output_dtype(self, dtype):
         """"f32" (default) or "f16": element type of the tensors forward() returns or fills."""
         self.out_dtype = dtype
@@ -288,7 +300,8 @@ class Conv:
     def forward(self, x, y=None):
         torch = self.torch
         N, C, K, H, W = self.shape
-        assert x.is_cuda and x.is_contiguous() and tuple(x.shape) == (N, C, H, W)
+        xs = (N, H, W, C) if getattr(self, "in_layout", "nchw") == "nhwc" else (N, C, H, W)
+        assert x.is_cuda and x.is_contiguous() and tuple(x.shape) == xs
         assert x.dtype == (torch.float16 if self.in_dtype == "f16" else torch.float32)
         ydt = torch.float16 if getattr(self, "out_dtype", "f32") == "f16" else torch.float32
         if y is None:

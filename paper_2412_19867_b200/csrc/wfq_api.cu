@@ -93,9 +93,9 @@ bool encode_tmap(CUtensorMap *map, CUtensorMapDataType dtype, int rank, const vo
             return false;
         encode = reinterpret_cast<EncodeFn>(fn);
     }
-    if (rank < 1 || rank > 3) return false;
-    cuuint64_t d[3], st[2];
-    cuuint32_t bx[3], estr[3] = {1u, 1u, 1u};
+    if (rank < 1 || rank > 4) return false;
+    cuuint64_t d[4], st[3];
+    cuuint32_t bx[4], estr[4] = {1u, 1u, 1u, 1u};
     for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; }
     for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
     CUresult r = encode(map, dtype, (cuuint32_t)rank, const_cast<void *>(base), d, st, bx, estr,
@@ -191,6 +191,17 @@ wfq_status_t wfq_plan_set_input_dtype(wfq_plan_t *plan, wfq_dtype_t dtype)
     return WFQ_OK;
 }
 
+wfq_status_t wfq_plan_set_input_layout(wfq_plan_t *plan, wfq_layout_t layout)
+{
+    if (!plan || (layout != WFQ_NCHW && layout != WFQ_NHWC)) return WFQ_ERR_INVALID_ARG;
+    if (layout == WFQ_NHWC && plan->fq_input) return WFQ_ERR_UNSUPPORTED;   // integer input transform: NCHW only
+    plan->in_nhwc = layout == WFQ_NHWC;
+    plan->tmap_xn_base = nullptr;
+    for (int i = 0; i < 2; ++i)
+        if (plan->sub[i]) { plan->sub[i]->in_nhwc = plan->in_nhwc; plan->sub[i]->tmap_xn_base = nullptr; }
+    return WFQ_OK;
+}
+
 wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_activation_t act)
 {
     if (!plan) return WFQ_ERR_INVALID_ARG;
@@ -220,7 +231,7 @@ wfq_status_t wfq_plan_set_full_quant(wfq_plan_t *plan, int quant_input, wfq_y_qu
     if (!plan) return WFQ_ERR_INVALID_ARG;
     if (quant_input != 0 && quant_input != 1) return WFQ_ERR_INVALID_ARG;
     if (y_mode != WFQ_Y_FP32 && y_mode != WFQ_Y_TILE && y_mode != WFQ_Y_ROW) return WFQ_ERR_INVALID_ARG;
-    if (quant_input && (plan->geo.gs % 32 != 0 || plan->geo.gs > 256)) return WFQ_ERR_UNSUPPORTED;
+    if (quant_input && (plan->geo.gs % 32 != 0 || plan->geo.gs > 256 || plan->in_nhwc)) return WFQ_ERR_UNSUPPORTED;
     plan->fq_input = quant_input != 0;
     plan->fq_output = (int)y_mode;
     for (int i = 0; i < 2; ++i)
@@ -493,6 +504,7 @@ static wfq_status_t setup_host_pipeline(wfq_plan *plan)
         wfq_plan *q = plan->sub[s];
         wfq_plan_set_input_dtype(q, plan->in_dtype);
         q->k1_choice = plan->k1_choice;
+        q->in_nhwc = plan->in_nhwc;
         // same orientation of the contraction as the whole batch: identical arithmetic
         q->gemm_swap = plan->gemm_swap;
         q->gemm_bn = plan->gemm_bn;

@@ -27,6 +27,7 @@
 #include <cuda_fp16.h>
 
 #include "wfq_internal.h"
+#include "wfq_ptx.cuh"
 
 namespace wfq {
 namespace {
@@ -109,6 +110,9 @@ __device__ __forceinline__ void bt_1d(const float2 (&d)[8], float2 (&r)[8])
     r[5] = __fadd2_rn(f, g);
     r[6] = __ffma2_rn(f2(-1.f), g, f);
 }
+
+__device__ __forceinline__ float to_float32(float v) { return v; }
+__device__ __forceinline__ float to_float32(__half v) { return __half2float(v); }
 
 // ---- patch load from the staged strip ---------------------------------------------
 // `ch` points at the channel's plane in smem; `col0` is the (even) smem column whose
@@ -368,6 +372,79 @@ __device__ __forceinline__ void group_scale(float amax, float &scale, float &inv
     inv = nz ? __fdiv_rn(127.f, amax) : 0.f;
 }
 
+// ---- phase 2 of a work item: quantize, one (tile, group, position) per thread -------------
+// Zs holds the transformed values of `ntile` tiles as [tile][position][CB + 4] fp32; the item is
+// tiles tw0 .. of tile row `srow` (= image * TH + tile row) and channels c_base .. c_base + CB.
+template <int P, int GSR, int SPLIT>
+__device__ __forceinline__ void quantize_item(const float *__restrict__ Zs, int CBP, int ntile, int ng, int gs,
+                                              int srow, int tw0, int c_base, const Geometry &g,
+                                              const ScaleTables &tab, int8_t *__restrict__ Xq,
+                                              float *__restrict__ sX)
+{
+    // X = Z * (caller's per-position factor) is formed here, one rounding, as the
+    // quantizer's input; then abs-max, scale, reciprocal and codes.
+    const int g_base = c_base / gs;
+    if constexpr (GSR > 0) {
+        // whole warps walk the loop so that the lanes sharing a group can shuffle
+        const int tasks = ntile * ng * P * SPLIT;
+        for (int base = 0; base < tasks; base += K1_THREADS) {
+            const int task = base + (int)threadIdx.x;
+            const bool act = task < tasks;          // the lanes of a group are all in or all out
+            const int tk = act ? task : 0;
+            const int part = tk % SPLIT, rest = tk / SPLIT;
+            const int q = rest / P, p = rest - q * P;
+            const int tl = q / ng, grp = q - tl * ng;
+            const int t = srow * g.TW + tw0 + tl;
+            const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs +
+                                                                 part * GSR);
+            int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs + part * GSR;
+            const float sp = tab.in_scale[p], sl = tab.in_scale_lo[p];
+            const float2 sp2 = make_float2(sp, sp), sl2 = make_float2(sl, sl);
+            float4 v[GSR / 4];
+            float amax = 0.f;
+#pragma unroll
+            for (int k = 0; k < GSR / 4; ++k) {
+                v[k] = scale4(src[k], sp2, sl2);
+                amax = absmax4(amax, v[k]);
+            }
+            if constexpr (SPLIT >= 2) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+            if constexpr (SPLIT >= 4) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+            float scale, inv;
+            group_scale(amax, scale, inv);
+            if (act) {
+#pragma unroll
+                for (int k = 0; k < GSR / 32; ++k)        // 32 codes = one full sector per store
+                    st_global_v8_b32(dst + 32 * k, codes4(v[8 * k], inv), codes4(v[8 * k + 1], inv),
+                                     codes4(v[8 * k + 2], inv), codes4(v[8 * k + 3], inv),
+                                     codes4(v[8 * k + 4], inv), codes4(v[8 * k + 5], inv),
+                                     codes4(v[8 * k + 6], inv), codes4(v[8 * k + 7], inv));
+                if (part == 0) sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
+            }
+        }
+    } else {
+        const int tasks = ntile * ng * P;
+        for (int task = threadIdx.x; task < tasks; task += K1_THREADS) {
+            const int q = task / P, p = task - q * P;
+            const int tl = q / ng, grp = q - tl * ng;
+            const int t = srow * g.TW + tw0 + tl;
+            const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs);
+            int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
+            const float sp = tab.in_scale[p], sl = tab.in_scale_lo[p];
+            const float2 sp2 = make_float2(sp, sp), sl2 = make_float2(sl, sl);
+            float scale, inv;
+            float amax = 0.f;
+            for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2, sl2));
+            group_scale(amax, scale, inv);
+            for (int k = 0; k < gs / 32; ++k)
+                st_global_v8_b32(dst + 32 * k, codes4(scale4(src[8 * k], sp2, sl2), inv),
+                                 codes4(scale4(src[8 * k + 1], sp2, sl2), inv), codes4(scale4(src[8 * k + 2], sp2, sl2), inv),
+                                 codes4(scale4(src[8 * k + 3], sp2, sl2), inv), codes4(scale4(src[8 * k + 4], sp2, sl2), inv),
+                                 codes4(scale4(src[8 * k + 5], sp2, sl2), inv), codes4(scale4(src[8 * k + 6], sp2, sl2), inv),
+                                 codes4(scale4(src[8 * k + 7], sp2, sl2), inv));
+            sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
+        }
+    }}
+
 // ---- the kernel ----------------------------------------------------------------------
 // GSR > 0: channels a thread holds in registers during phase 2 (32 or 64); a group is GSR *
 // SPLIT channels, SPLIT neighbouring lanes share it and exchange their abs-max by shuffle.
@@ -451,71 +528,120 @@ input_transform_kernel(const Tin *__restrict__ x, int8_t *__restrict__ Xq,
         __syncthreads();
         if (!prm.dbuf && next < prm.items) stage_item(next, 0);   // the strip buffer is free: refill it now
 
-        // ---- phase 2: quantize, one (tile, group, position) per thread -------------------
-        // X = Z * (caller's per-position factor) is formed here, one rounding, as the
-        // quantizer's input; then abs-max, scale, reciprocal and codes.
-        const int g_base = c_base / gs;
-        if constexpr (GSR > 0) {
-            // whole warps walk the loop so that the lanes sharing a group can shuffle
-            const int tasks = ntile * ng * P * SPLIT;
-            for (int base = 0; base < tasks; base += K1_THREADS) {
-                const int task = base + (int)threadIdx.x;
-                const bool act = task < tasks;          // the lanes of a group are all in or all out
-                const int tk = act ? task : 0;
-                const int part = tk % SPLIT, rest = tk / SPLIT;
-                const int q = rest / P, p = rest - q * P;
-                const int tl = q / ng, grp = q - tl * ng;
-                const int t = srow * g.TW + tw0 + tl;
-                const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs +
-                                                                     part * GSR);
-                int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs + part * GSR;
-                const float sp = tab.in_scale[p], sl = tab.in_scale_lo[p];
-                const float2 sp2 = make_float2(sp, sp), sl2 = make_float2(sl, sl);
-                float4 v[GSR / 4];
-                float amax = 0.f;
-#pragma unroll
-                for (int k = 0; k < GSR / 4; ++k) {
-                    v[k] = scale4(src[k], sp2, sl2);
-                    amax = absmax4(amax, v[k]);
-                }
-                if constexpr (SPLIT >= 2) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-                if constexpr (SPLIT >= 4) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-                float scale, inv;
-                group_scale(amax, scale, inv);
-                if (act) {
-#pragma unroll
-                    for (int k = 0; k < GSR / 32; ++k)        // 32 codes = one full sector per store
-                        st_global_v8_b32(dst + 32 * k, codes4(v[8 * k], inv), codes4(v[8 * k + 1], inv),
-                                         codes4(v[8 * k + 2], inv), codes4(v[8 * k + 3], inv),
-                                         codes4(v[8 * k + 4], inv), codes4(v[8 * k + 5], inv),
-                                         codes4(v[8 * k + 6], inv), codes4(v[8 * k + 7], inv));
-                    if (part == 0) sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
-                }
-            }
-        } else {
-            const int tasks = ntile * ng * P;
-            for (int task = threadIdx.x; task < tasks; task += K1_THREADS) {
-                const int q = task / P, p = task - q * P;
-                const int tl = q / ng, grp = q - tl * ng;
-                const int t = srow * g.TW + tw0 + tl;
-                const float4 *src = reinterpret_cast<const float4 *>(Zs + (size_t)(tl * P + p) * CBP + grp * gs);
-                int8_t *dst = Xq + ((size_t)p * g.T + t) * g.C + c_base + grp * gs;
-                const float sp = tab.in_scale[p], sl = tab.in_scale_lo[p];
-                const float2 sp2 = make_float2(sp, sp), sl2 = make_float2(sl, sl);
-                float scale, inv;
-                float amax = 0.f;
-                for (int k = 0; k < gs / 4; ++k) amax = absmax4(amax, scale4(src[k], sp2, sl2));
-                group_scale(amax, scale, inv);
-                for (int k = 0; k < gs / 32; ++k)
-                    st_global_v8_b32(dst + 32 * k, codes4(scale4(src[8 * k], sp2, sl2), inv),
-                                     codes4(scale4(src[8 * k + 1], sp2, sl2), inv), codes4(scale4(src[8 * k + 2], sp2, sl2), inv),
-                                     codes4(scale4(src[8 * k + 3], sp2, sl2), inv), codes4(scale4(src[8 * k + 4], sp2, sl2), inv),
-                                     codes4(scale4(src[8 * k + 5], sp2, sl2), inv), codes4(scale4(src[8 * k + 6], sp2, sl2), inv),
-                                     codes4(scale4(src[8 * k + 7], sp2, sl2), inv));
-                sX[((size_t)p * g.G + g_base + grp) * g.Ts + t] = scale;
-            }
-        }
+        quantize_item<P, GSR, SPLIT>(Zs, CBP, ntile, ng, gs, srow, tw0, c_base, g, tab, Xq, sX);
         __syncthreads();   // Z and this strip buffer are free again
+    }
+}
+
+// ---- the same for an NHWC input ---------------------------------------------------------
+// x[N][H][W][C]: the channels are innermost, so the strip of a work item is one 4-D TMA box
+// {CB channels, TB * m + 2 columns, n rows, 1 image} (zero fill outside the image, no alignment
+// condition on the row or column it starts at) and lands as [row][column][channel]; a thread
+// reads its patch with the lanes along the channels (no bank conflicts, no realignment).  One
+// thread issues the copy of an item as soon as the buffer it goes to has been read; everything
+// else is the kernel above: transform, [tile][position][channel] array, quantize_item.
+struct K1NhwcShared {
+    uint64_t full[2];        // the strip of a buffer has landed
+    volatile int abort;
+};
+
+template <int M, typename Tin, int GSR, int SPLIT>
+__global__ void __launch_bounds__(K1_THREADS, 4)
+input_transform_nhwc_kernel(const __grid_constant__ CUtensorMap tmx, int8_t *__restrict__ Xq,
+                            float *__restrict__ sX, Geometry g, ScaleTables tab, K1Params prm, int *status,
+                            long long wait_cycles)
+{
+    constexpr int NN = M + 2;
+    constexpr int P = NN * NN;
+    extern __shared__ __align__(16) unsigned char smem_dyn[];
+    __shared__ K1NhwcShared sh;
+    // a TMA destination must be 128-byte aligned; the dynamic part starts wherever the static part
+    // ends, so the strips start at the next multiple of 128 (the launch adds 128 bytes for this)
+    unsigned char *smem_raw = reinterpret_cast<unsigned char *>(
+        (reinterpret_cast<uintptr_t>(smem_dyn) + 127) & ~(uintptr_t)127);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    float *Zs = reinterpret_cast<float *>(smem_raw + (1 + prm.dbuf) * prm.strip_bytes);   // [tile][position][CBP]
+    const int CBP = prm.CB + 4;
+    const int WB = prm.TB * M + 2;                     // columns of the box
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int NWARP = K1_THREADS / 32;
+    const int cb32 = prm.CB >> 5;
+    const int gs = GSR > 0 ? GSR * SPLIT : g.gs;
+    const int ng = prm.CB / gs;
+    const WaitCtx ctx{&sh.abort, status, wait_cycles};
+    const uint32_t box_bytes = (uint32_t)(NN * WB * prm.CB * (int)sizeof(Tin));
+
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_u32(&sh.full[0]), 1);
+        ptx::mbar_init(ptx::smem_u32(&sh.full[1]), 1);
+        sh.abort = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmx);
+    }
+    __syncthreads();
+
+    // thread 0 only
+    auto issue = [&](int item, int buf) {
+        const int cblk = item % prm.NCB, rest = item / prm.NCB;
+        const int srow = rest / prm.NCH, chunk = rest - srow * prm.NCH;
+        const int img = srow / g.TH, th = srow - img * g.TH;
+        const uint32_t bar = ptx::smem_u32(&sh.full[buf]);
+        ptx::mbar_arrive_expect_tx(bar, box_bytes);
+        ptx::tma_load_4d(ptx::smem_u32(smem_raw + buf * prm.strip_bytes), &tmx, bar, cblk * prm.CB,
+                         chunk * prm.TB * M - 1, th * M - 1, img);
+    };
+
+    const int stride = (int)gridDim.x;
+    int item = blockIdx.x;
+    int issued = 0;                                     // items whose copy has been issued (thread 0)
+    if (threadIdx.x == 0) {
+        if (item < prm.items) { issue(item, 0); ++issued; }
+        if (prm.dbuf && item + stride < prm.items) { issue(item + stride, 1); ++issued; }
+    }
+    bool ok = true;
+    int it = 0;
+    for (; item < prm.items; ++it, item += stride) {
+        const int buf = prm.dbuf ? (it & 1) : 0;
+        const uint32_t parity = (uint32_t)(prm.dbuf ? (it >> 1) : it) & 1u;
+        ok = wait_bounded(ptx::smem_u32(&sh.full[buf]), parity, ctx, kWaitStripFull);
+        if (!ok) break;
+
+        const Tin *strip = reinterpret_cast<const Tin *>(smem_raw + buf * prm.strip_bytes);
+        const int cblk = item % prm.NCB, rest = item / prm.NCB;
+        const int srow = rest / prm.NCH, chunk = rest - srow * prm.NCH;
+        const int tw0 = chunk * prm.TB;
+        const int ntile = min(prm.TB, g.TW - tw0);
+        const int c_base = cblk * prm.CB;
+
+        // ---- phase 1: transform, one (tile, channel) per thread ----------------------
+        for (int wt = warp; wt < ntile * cb32; wt += NWARP) {
+            const int tl = wt / cb32;
+            const int c = (wt - tl * cb32) * 32 + lane;
+            float d[NN][NN];
+            const Tin *src = strip + (size_t)(tl * M) * prm.CB + c;
+#pragma unroll
+            for (int a = 0; a < NN; ++a)
+#pragma unroll
+                for (int b = 0; b < NN; ++b) d[a][b] = to_float32(src[(a * WB + b) * prm.CB]);
+            transform_patch<NN>(d, Zs + (size_t)tl * P * CBP + c, CBP);
+        }
+        __syncthreads();
+        // the strip buffer has been read: the item that uses it next may be copied now
+        if (threadIdx.x == 0) {
+            const int nxt = item + (prm.dbuf ? 2 : 1) * stride;
+            if (nxt < prm.items) { issue(nxt, buf); ++issued; }
+        }
+        quantize_item<P, GSR, SPLIT>(Zs, CBP, ntile, ng, gs, srow, tw0, c_base, g, tab, Xq, sX);
+        __syncthreads();   // Z is free again
+    }
+    if (!ok && threadIdx.x == 0) {
+        // a copy never arrived: give the ones still in flight a bounded time to land before the
+        // shared memory goes away (copies issued: `issued`, consumed: `it`)
+        for (int k = it; k < issued; ++k) {
+            const int b = prm.dbuf ? (k & 1) : 0;
+            drain(ptx::smem_u32(&sh.full[b]), (uint32_t)(prm.dbuf ? (k >> 1) : k) & 1u, wait_cycles / 16);
+        }
     }
 }
 
@@ -557,8 +683,42 @@ cudaError_t launch_k1(const wfq_plan &plan, const void *x_dev, cudaStream_t stre
                               plan.ws.Xq, plan.ws.sX, plan.geo, plan.tables, prm);
 }
 
+template <int M, typename Tin, int GSR, int SPLIT>
+int k1n_resident(size_t smem)
+{
+    return resident_ctas_per_sm(input_transform_nhwc_kernel<M, Tin, GSR, SPLIT>, K1_THREADS, smem, 32);
+}
+
+template <int M, typename Tin, int GSR, int SPLIT>
+cudaError_t k1n_setup()
+{
+    auto kern = input_transform_nhwc_kernel<M, Tin, GSR, SPLIT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                (int)cudaSharedmemCarveoutMaxShared);
+}
+
+template <int M, typename Tin, int GSR, int SPLIT>
+cudaError_t launch_k1n(const wfq_plan &plan, cudaStream_t stream)
+{
+    const K1Params &prm = plan.k1n;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)prm.grid);
+    cfg.blockDim = dim3(K1_THREADS);
+    cfg.dynamicSmemBytes = prm.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, input_transform_nhwc_kernel<M, Tin, GSR, SPLIT>, plan.tmap_xn, plan.ws.Xq,
+                              plan.ws.sX, plan.geo, plan.tables, prm, plan.status, plan.wait_cycles);
+}
+
 // What to do with the instantiation that serves (m, dtype, group size).
-enum K1Op { kK1Launch, kK1Resident, kK1Setup };
+enum K1Op { kK1Launch, kK1Resident, kK1Setup, kK1nLaunch, kK1nResident, kK1nSetup };
 
 template <int M, typename Tin>
 long long k1_by_gs(K1Op op, int gs, const wfq_plan *plan, const void *x, cudaStream_t s, size_t smem)
@@ -567,7 +727,10 @@ long long k1_by_gs(K1Op op, int gs, const wfq_plan *plan, const void *x, cudaStr
     switch (op) {                                                                      \
         case kK1Launch: return (long long)launch_k1<M, Tin, GSR, SPLIT>(*plan, x, s);  \
         case kK1Resident: return k1_resident<M, Tin, GSR, SPLIT>(smem);                \
-        default: return (long long)k1_setup<M, Tin, GSR, SPLIT>();                     \
+        case kK1Setup: return (long long)k1_setup<M, Tin, GSR, SPLIT>();               \
+        case kK1nLaunch: return (long long)launch_k1n<M, Tin, GSR, SPLIT>(*plan, s);   \
+        case kK1nResident: return k1n_resident<M, Tin, GSR, SPLIT>(smem);              \
+        default: return (long long)k1n_setup<M, Tin, GSR, SPLIT>();                    \
     }
     if (gs == 32) { WFQ_K1_CASE(32, 1) }
     if (gs == 64) { WFQ_K1_CASE(64, 1) }
@@ -635,6 +798,43 @@ void plan_k1(wfq_plan &plan, K1Params &prm, bool vec16)
 
 }  // namespace
 
+// The same for the NHWC kernel: the strip is the dense TMA box [n][TB * m + 2][CB].
+static void plan_k1_nhwc(wfq_plan &plan)
+{
+    const Geometry &g = plan.geo;
+    const bool f16 = plan.in_dtype == WFQ_F16;
+    const int NN = g.n, P = g.P, M = g.m;
+    const int esz = f16 ? 2 : 4;
+    K1Params &prm = plan.k1n;
+    prm = plan.k1;
+    prm.vec16 = 0;
+    prm.TB = (K1_WP - 3) / M;
+    prm.CB = g.gs;
+    if (g.gs == 32 && g.C % 64 == 0) prm.CB = 64;
+    auto strip = [&]() { return ((NN * (prm.TB * M + 2) * prm.CB * esz + 127) / 128) * 128; };
+    auto smem_bytes = [&]() {     // 128 bytes of slack for the alignment of the strips
+        return 128 + (1 + prm.dbuf) * (size_t)strip() + (size_t)prm.TB * P * (prm.CB + 4) * sizeof(float);
+    };
+    prm.dbuf = 0;
+    while (prm.TB > 1 && smem_bytes() > 113 * 1024) --prm.TB;
+    prm.NCH = (g.TW + prm.TB - 1) / prm.TB;
+    prm.TB = (g.TW + prm.NCH - 1) / prm.NCH;
+    {
+        const size_t per_sm = 226 * 1024, one = smem_bytes() + 1024;
+        const size_t two = one + strip();
+        const size_t n1 = per_sm / one < 4 ? per_sm / one : 4, n2 = per_sm / two < 4 ? per_sm / two : 4;
+        if (n2 >= 1 && n2 == n1) prm.dbuf = 1;
+    }
+    prm.strip_bytes = strip();
+    prm.CS = 0;
+    prm.smem = (int)smem_bytes();
+    prm.NCB = g.C / prm.CB;
+    prm.items = g.N * g.TH * prm.NCH * prm.NCB;
+    const int per_sm = (int)k1_op(kK1nResident, M, f16, g.gs, nullptr, nullptr, nullptr, (size_t)prm.smem);
+    const int resident = per_sm * (plan.sm_count > 0 ? plan.sm_count : 1);
+    prm.grid = prm.items < resident ? prm.items : resident;
+}
+
 // Work-item shape, shared-memory layout and grid of the cp.async kernel for this plan: one set
 // with 4-byte (or 2-byte) copies for any x, and where fp16 rows are whole 16-byte pieces (W a
 // multiple of 8) a second one with 16-byte copies, used when x is 16-byte aligned.
@@ -643,6 +843,8 @@ void plan_input_transform(wfq_plan &plan)
     plan_k1(plan, plan.k1, false);
     plan.k1v = plan.k1;
     if (plan.in_dtype == WFQ_F16 && plan.geo.W % 8 == 0) plan_k1(plan, plan.k1v, true);
+    plan_k1_nhwc(plan);
+    plan.tmap_xn_base = nullptr;
 }
 
 cudaError_t setup_input_transform()
@@ -653,6 +855,8 @@ cudaError_t setup_input_transform()
             for (int gs : sizes) {
                 cudaError_t e = (cudaError_t)k1_op(kK1Setup, m, f16 != 0, gs, nullptr, nullptr, nullptr, 0);
                 if (e != cudaSuccess) return e;
+                e = (cudaError_t)k1_op(kK1nSetup, m, f16 != 0, gs, nullptr, nullptr, nullptr, 0);
+                if (e != cudaSuccess) return e;
             }
     return cudaSuccess;
 }
@@ -660,6 +864,24 @@ cudaError_t setup_input_transform()
 cudaError_t launch_input_transform(wfq_plan &plan, const void *x_dev, cudaStream_t stream)
 {
     const Geometry &g = plan.geo;
+    if (plan.in_nhwc) {
+        // x[N][H][W][C] as a 4-D tensor (C, W, H, N) with boxes of one work item's strip
+        if ((reinterpret_cast<uintptr_t>(x_dev) & 15u) != 0) return cudaErrorInvalidValue;
+        if (plan.tmap_xn_base != x_dev) {
+            const unsigned long long esz = plan.in_dtype == WFQ_F16 ? 2 : 4;
+            const unsigned long long dims[4] = {(unsigned long long)g.C, (unsigned long long)g.W,
+                                                (unsigned long long)g.H, (unsigned long long)g.N};
+            const unsigned long long strides[3] = {(unsigned long long)g.C * esz, (unsigned long long)g.W * g.C * esz,
+                                                   (unsigned long long)g.H * g.W * g.C * esz};
+            const unsigned box[4] = {(unsigned)plan.k1n.CB, (unsigned)(plan.k1n.TB * g.m + 2), (unsigned)g.n, 1u};
+            if (!encode_tmap(&plan.tmap_xn, plan.in_dtype == WFQ_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                                      : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                             4, x_dev, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+                return cudaErrorInvalidValue;
+            plan.tmap_xn_base = x_dev;
+        }
+        return (cudaError_t)k1_op(kK1nLaunch, g.m, plan.in_dtype == WFQ_F16, g.gs, &plan, x_dev, stream, 0);
+    }
     // tensor-core kernel: fp16 input that a TMA tensor map (16-byte aligned base) can describe
     // (automatic = the cp.async kernel: the tensor-core one measured no faster on any configured layer)
     if (plan.k1tc.use && plan.k1_choice == 2 && (reinterpret_cast<uintptr_t>(x_dev) & 15u) == 0) {

@@ -122,6 +122,10 @@ struct wfq_plan {
     // launch parameters derived from the geometry, the dtype and the device (plan_launches)
     wfq::K1Params k1;          // 4-byte (or 2-byte) copies: any x
     wfq::K1Params k1v;         // 16-byte copies where the layer allows them (vec16 set), else a copy of k1
+    wfq::K1Params k1n;         // NHWC input: one TMA box per work item
+    bool in_nhwc = false;      // x is [N][H][W][C] instead of [N][C][H][W]
+    CUtensorMap tmap_xn;       // the NHWC input as (C, W, H, N)
+    const void *tmap_xn_base = nullptr;   // x pointer tmap_xn was encoded for
     wfq::K1TcPlan k1tc;
     CUtensorMap tmap_x;        // the input tensor as the tensor-core input transform stages it
     const void *tmap_x_base = nullptr;   // x pointer tmap_x was encoded for

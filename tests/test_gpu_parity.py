@@ -207,6 +207,48 @@ def test_contraction_shapes_agree(layer):
     conv.close()
 
 
+@pytest.mark.parametrize("layer", [
+    Layer(1, 64, 32, 13, 11, 6, 64, "f16", "silu_outlier", "kaiming_chan", 9, 8, 1),      # ragged edges
+    Layer(3, 192, 32, 20, 24, 4, 32, "f32", "gauss_outlier", "gauss_chan", 9, 8, 2),      # fp32, two groups per item
+    Layer(2, 256, 32, 28, 28, 6, 128, "f16", "relu_heavy", "kaiming", 9, 8, 3),           # two lanes per group
+    Layer(1, 192, 32, 12, 24, 4, 96, "f16", "silu_outlier", "kaiming_chan", 9, 8, 4),     # generic group size
+    Layer(2, 128, 48, 56, 56, 6, 64, "f16", "relu_heavy", "kaiming", 9, 8, 5),            # several items per CTA
+    Layer(1, 512, 32, 16, 16, 4, 256, "f16", "silu_outlier", "kaiming_chan", 9, 8, 6),    # four lanes per group
+], ids=lambda L: L.name)
+def test_nhwc_input_matches_nchw(layer):
+    """x given as [N][H][W][C] (TMA-staged input transform): codes and scales of stage 1 and the
+    final output equal the NCHW path's bit for bit, and the oracle's within the usual bars;
+    also through the host-buffer entry point, and back to NCHW on the same plan."""
+    import torch
+    from oracle import oracle as orc
+    from paper_2412_19867_b200 import binding as b
+    from tests import gpu_util as gu
+    L = layer
+    conv, (x, w, sB, sG) = gu.make_conv(L)
+    xd = torch.from_numpy(x).to("cuda:0")
+    xn = xd.permute(0, 2, 3, 1).contiguous()
+    y0 = conv.forward(xd)
+    xq0 = conv.buffer(b.WFQ_BUF_XQ).clone()
+    sx0 = conv.buffer(b.WFQ_BUF_SX)[:, :, :conv.T].clone()
+    conv.set_input_layout("nhwc")
+    conv.buffer(b.WFQ_BUF_XQ).fill_(99)
+    y1 = conv.forward(xn)
+    conv.check_status()
+    assert torch.equal(conv.buffer(b.WFQ_BUF_XQ), xq0)
+    assert torch.equal(conv.buffer(b.WFQ_BUF_SX)[:, :, :conv.T], sx0)
+    assert torch.equal(y0, y1)
+    ref = orc.wfq(x, w[:1], L.m, L.gs, sB=sB, sG=sG)
+    gu.codes_close(xq0.cpu().numpy(), ref.Xq)
+    yh = torch.empty(y0.shape, dtype=torch.float32).pin_memory()
+    conv.forward_host(xn.cpu().pin_memory(), yh)
+    assert torch.equal(yh, y0.cpu())
+    with pytest.raises(b.WfqError):
+        b.wfq_plan_set_full_quant(conv.plan, 1, b.WFQ_Y_FP32)
+    conv.set_input_layout("nchw")
+    assert torch.equal(conv.forward(xd), y0)
+    conv.close()
+
+
 def test_filters_export_and_import():
     """A plan made ready from an exported blob computes what the plan that prepared the filters
     computes (also for another batch and image size, and in the fully quantized mode); a blob
