@@ -106,7 +106,9 @@ typedef enum {
 /*
  * Create a plan for one layer: x[N][C][H][W] -> y[N][K][H][W] evaluated as F(m,3)
  * (Section 3.1: output tile m x m, filter r x r, input tile (m+r-1)^2).
- * Supported: r = 3; m in {4, 6}; bits = 8; group_size a multiple of 32, at most 256,
+ * Supported: r = 3; m in {2, 4, 6} (F(4,3) and F(6,3) are the paper's tiles; F(2,3) is the textbook
+ * tile with the matrices B^T = [1 0 -1 0; 0 1 1 0; 0 -1 1 0; 0 1 0 -1], G = [1 0 0; 1/2 1/2 1/2;
+ * 1/2 -1/2 1/2; 0 0 1], A^T = [1 1 1 0; 0 1 -1 -1] as its standard scaling); bits = 8; group_size a multiple of 32, at most 256,
  * dividing C; N, C, K, H, W >= 1; P*T*C, P*K*C and N*K*H*W below 2^31.
  * Returns WFQ_ERR_INVALID_ARG for NULL/non-positive arguments and
  * WFQ_ERR_UNSUPPORTED for anything else outside this set.  Synchronous, host-only
@@ -222,7 +224,7 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
  *   sG_host      host, m+2 floats, diagonal of S_G; NULL = standard scales
  *   wq_dev       device, int8 [P][K][C], caller-owned                    (output)
  *   sw_dev       device, fp32 [P][C/group_size][K], caller-owned         (output)
- *   m in {4,6}; group_size a multiple of 32, at most 256, dividing C.
+ *   m in {2,4,6}; group_size a multiple of 32, at most 256, dividing C.
  *
  * Limit: (m+2)^2 * K * C <= WFQ_STATIC_SCRATCH_FLOATS, otherwise
  * WFQ_ERR_SCRATCH_TOO_SMALL is returned and nothing is launched.  Other argument errors

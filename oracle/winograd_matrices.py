@@ -7,7 +7,9 @@ imports it and carries its own hand-written tables.
 Everything here is exact rational arithmetic (``fractions.Fraction``) and follows
 the paper's supplementary section "Standard Winograd transforms":
 
-* the polynomial points ``(f_i, g_i)`` of F(4,3) and F(6,3),
+* the polynomial points ``(f_i, g_i)`` of F(4,3) and F(6,3) (and, beyond the paper, of the
+  textbook F(2,3): points 0, 1, -1, infinity, scales chosen so that the matrices are the
+  familiar ones of the fast-convolution literature),
 * the Vandermonde matrix ``V_{a x b}[i][j] = f_i**j * g_i**(b-1-j)``,
 * ``A^T = V_{n x m}^T S_A``      (Eq. ``scale_a``),
 * ``B^T = S_B V_{n x n}^{-T}``   (Eq. ``scale_b``),
@@ -25,6 +27,7 @@ R = 3  # filter size; the paper uses F(m, 3) throughout
 
 # Polynomial points (f_i, g_i); the last one, (1, 0), is the point at infinity.
 POINTS = {
+    2: [(Fr(0), Fr(1)), (Fr(1), Fr(1)), (Fr(-1), Fr(1)), (Fr(1), Fr(0))],
     4: [(Fr(0), Fr(1)), (Fr(1), Fr(1)), (Fr(-1), Fr(1)),
         (Fr(2), Fr(1)), (Fr(-2), Fr(1)), (Fr(1), Fr(0))],
     6: [(Fr(0), Fr(1)), (Fr(1), Fr(1)), (Fr(-1), Fr(1)), (Fr(2), Fr(1)),
@@ -33,6 +36,9 @@ POINTS = {
 
 # Standard scaling factors printed next to the points.
 STANDARD_SCALES = {
+    2: dict(SA=[Fr(1), Fr(1), Fr(1), Fr(-1)],
+            SB=[Fr(1), Fr(2), Fr(2), Fr(-1)],
+            SG=[Fr(1), Fr(1, 2), Fr(1, 2), Fr(1)]),
     4: dict(SA=[Fr(1)] * 6,
             SB=[Fr(4), Fr(-6), Fr(-6), Fr(24), Fr(24), Fr(1)],
             SG=[Fr(1, 4), Fr(-1, 6), Fr(-1, 6), Fr(1, 24), Fr(1, 24), Fr(1)]),

@@ -13,6 +13,8 @@ namespace {
 // Standard scale vectors of the paper's supplementary ("Standard Winograd
 // transforms"): used when the caller passes NULL, and as the reference the kernels'
 // hard-coded integer/rational transform matrices are scaled by.
+const double kStdSB2[4] = {1.0, 2.0, 2.0, -1.0};          // F(2,3): the textbook matrices
+const double kStdSG2[4] = {1.0, 0.5, 0.5, 1.0};
 const double kStdSB4[6] = {4.0, -6.0, -6.0, 24.0, 24.0, 1.0};
 const double kStdSG4[6] = {1.0 / 4, -1.0 / 6, -1.0 / 6, 1.0 / 24, 1.0 / 24, 1.0};
 const double kStdSB6[8] = {1.0, -4.5, -4.5, 90.0, 90.0, 45.0 / 32, 45.0 / 32, 1.0};
@@ -145,7 +147,7 @@ wfq_status_t wfq_plan_create(wfq_plan_t **out, int N, int C, int K, int H, int W
     *out = nullptr;
     if (N < 1 || C < 1 || K < 1 || H < 1 || W < 1 || m < 1 || r < 1 || group_size < 1 || bits < 1)
         return WFQ_ERR_INVALID_ARG;
-    if (r != 3 || (m != 4 && m != 6) || bits != 8) return WFQ_ERR_UNSUPPORTED;
+    if (r != 3 || (m != 2 && m != 4 && m != 6) || bits != 8) return WFQ_ERR_UNSUPPORTED;
     if (group_size % 32 != 0 || group_size > 256 || C % group_size != 0)
         return WFQ_ERR_UNSUPPORTED;
 
@@ -263,7 +265,7 @@ wfq_status_t wfq_plan_set_workspace(wfq_plan_t *plan, void *dev_ptr, size_t byte
 static void fill_scale_tables(wfq_plan *plan)
 {
     const wfq::Geometry &g = plan->geo;
-    const double *stdB = g.m == 4 ? kStdSB4 : kStdSB6;
+    const double *stdB = g.m == 2 ? kStdSB2 : g.m == 4 ? kStdSB4 : kStdSB6;
     for (int i = 0; i < g.n; ++i)
         for (int j = 0; j < g.n; ++j) {
             const double f = (plan->sB[i] / stdB[i]) * (plan->sB[j] / stdB[j]);
@@ -312,8 +314,8 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
 {
     if (!plan || !w_dev) return WFQ_ERR_INVALID_ARG;
     const wfq::Geometry &g = plan->geo;
-    const double *stdB = g.m == 4 ? kStdSB4 : kStdSB6;
-    const double *stdG = g.m == 4 ? kStdSG4 : kStdSG6;
+    const double *stdB = g.m == 2 ? kStdSB2 : g.m == 4 ? kStdSB4 : kStdSB6;
+    const double *stdG = g.m == 2 ? kStdSG2 : g.m == 4 ? kStdSG4 : kStdSG6;
     for (int i = 0; i < g.n; ++i) {
         const double b = sB_host ? (double)sB_host[i] : stdB[i];
         const double s = sG_host ? (double)sG_host[i] : stdG[i];

@@ -155,19 +155,20 @@ extern "C" wfq_status_t wfq_quantize_filters_static(const float *w_dev, int K, i
     using namespace wfq;
     if (!w_dev || !wq_dev || !sw_dev) return WFQ_ERR_INVALID_ARG;
     if (K < 1 || C < 1 || m < 1 || group_size < 1) return WFQ_ERR_INVALID_ARG;
-    if ((m != 4 && m != 6) || group_size % 32 != 0 || group_size > 256 || C % group_size != 0)
+    if ((m != 2 && m != 4 && m != 6) || group_size % 32 != 0 || group_size > 256 || C % group_size != 0)
         return WFQ_ERR_UNSUPPORTED;
     const int n = m + 2, P = n * n;
     const unsigned long long need = (unsigned long long)P * (unsigned long long)K * (unsigned long long)C;
     if (need > kStaticScratchFloats) return WFQ_ERR_SCRATCH_TOO_SMALL;
 
+    static const double std2[4] = {1.0, 0.5, 0.5, 1.0};
     static const double std4[6] = {1.0 / 4, -1.0 / 6, -1.0 / 6, 1.0 / 24, 1.0 / 24, 1.0};
     static const double std6[8] = {1.0, -2.0 / 9, -2.0 / 9, 1.0 / 90, 1.0 / 90, 32.0 / 45, 32.0 / 45, 1.0};
     GScales sg;
     for (int i = 0; i < kMaxN; ++i) {
         double v = 0.0;
         if (i < n) {
-            v = sG_host ? (double)sG_host[i] : (m == 4 ? std4[i] : std6[i]);
+            v = sG_host ? (double)sG_host[i] : (m == 2 ? std2[i] : m == 4 ? std4[i] : std6[i]);
             if (!std::isfinite(v) || v == 0.0) return WFQ_ERR_INVALID_ARG;
         }
         sg.s[i] = v;

@@ -259,9 +259,12 @@ output_transform_int_kernel(const float *__restrict__ Y, float *__restrict__ y, 
 }
 
 // Points of F(4,3) and F(6,3) (Section 3.1), the last one at infinity.
+const double kPoints2[3] = {0.0, 1.0, -1.0};
 const double kPoints4[5] = {0.0, 1.0, -1.0, 2.0, -2.0};
 const double kPoints6[7] = {0.0, 1.0, -1.0, 2.0, -2.0, 0.5, -0.5};
 // Standard-scaled B^T of the paper's supplementary and its row scales: V_B = diag(1 / s) B^T.
+const double kStdBT2[16] = {1, 0, -1, 0,   0, 1, 1, 0,   0, -1, 1, 0,   0, 1, 0, -1};
+const double kStdRow2[4] = {1.0, 2.0, 2.0, -1.0};
 const double kStdBT4[36] = {4, 0, -5, 0, 1, 0,   0, -4, -4, 1, 1, 0,   0, 4, -4, -1, 1, 0,
                             0, -2, -1, 2, 1, 0,  0, 2, -1, -2, 1, 0,   0, 4, 0, -5, 0, 1};
 const double kStdRow4[6] = {4.0, -6.0, -6.0, 24.0, 24.0, 1.0};
@@ -294,9 +297,9 @@ void build_full_quant_tables(wfq_plan &plan)
     const Geometry &g = plan.geo;
     const int n = g.n, m = g.m;
     FullQuantTables &tab = plan.fq;
-    const double *bt = m == 4 ? kStdBT4 : kStdBT6;
-    const double *row = m == 4 ? kStdRow4 : kStdRow6;
-    const double *pts = m == 4 ? kPoints4 : kPoints6;
+    const double *bt = m == 2 ? kStdBT2 : m == 4 ? kStdBT4 : kStdBT6;
+    const double *row = m == 2 ? kStdRow2 : m == 4 ? kStdRow4 : kStdRow6;
+    const double *pts = m == 2 ? kPoints2 : m == 4 ? kPoints4 : kPoints6;
     double BT[kMaxN * kMaxN], AT[kMaxN * kMaxN];
     // S_B V_B: V_B = V^{-T}, each entry the correctly rounded quotient of two exact numbers
     for (int i = 0; i < n; ++i)
@@ -341,11 +344,13 @@ cudaError_t launch_input_transform_int(const wfq_plan &plan, const void *x_dev, 
     float *sX = plan.ws.sX;
     if (plan.in_dtype == WFQ_F16) {
         const __half *x = static_cast<const __half *>(x_dev);
-        if (g.m == 4) input_transform_int_kernel<4, __half><<<grid, block, smem, stream>>>(x, Xq, sX, g, plan.fq);
+        if (g.m == 2) input_transform_int_kernel<2, __half><<<grid, block, smem, stream>>>(x, Xq, sX, g, plan.fq);
+        else if (g.m == 4) input_transform_int_kernel<4, __half><<<grid, block, smem, stream>>>(x, Xq, sX, g, plan.fq);
         else input_transform_int_kernel<6, __half><<<grid, block, smem, stream>>>(x, Xq, sX, g, plan.fq);
     } else {
         const float *x = static_cast<const float *>(x_dev);
-        if (g.m == 4) input_transform_int_kernel<4, float><<<grid, block, smem, stream>>>(x, Xq, sX, g, plan.fq);
+        if (g.m == 2) input_transform_int_kernel<2, float><<<grid, block, smem, stream>>>(x, Xq, sX, g, plan.fq);
+        else if (g.m == 4) input_transform_int_kernel<4, float><<<grid, block, smem, stream>>>(x, Xq, sX, g, plan.fq);
         else input_transform_int_kernel<6, float><<<grid, block, smem, stream>>>(x, Xq, sX, g, plan.fq);
     }
     return cudaGetLastError();
@@ -357,10 +362,12 @@ cudaError_t launch_output_transform_int(const wfq_plan &plan, float *y_dev, cuda
     const dim3 grid((unsigned)((g.T + 127) / 128), (unsigned)g.K), block(128);
     const float *Y = plan.ws.Y;
     if (plan.fq_output == 1) {
-        if (g.m == 4) output_transform_int_kernel<4, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
+        if (g.m == 2) output_transform_int_kernel<2, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
+        else if (g.m == 4) output_transform_int_kernel<4, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
         else output_transform_int_kernel<6, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
     } else {
-        if (g.m == 4) output_transform_int_kernel<4, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
+        if (g.m == 2) output_transform_int_kernel<2, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
+        else if (g.m == 4) output_transform_int_kernel<4, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
         else output_transform_int_kernel<6, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
     }
     return cudaGetLastError();

@@ -38,6 +38,15 @@ constexpr int K1_WPV = 24;       // the same where rows are copied in aligned 16
 
 // ---- 1-D input transforms with the standard B^T ------------------------------------
 
+// F(2,3) (the textbook matrices): rows [1,0,-1,0] [0,1,1,0] [0,-1,1,0] [0,1,0,-1]
+__device__ __forceinline__ void bt_1d(const float (&d)[4], float (&r)[4])
+{
+    r[0] = d[0] - d[2];
+    r[1] = d[1] + d[2];
+    r[2] = d[2] - d[1];
+    r[3] = d[1] - d[3];
+}
+
 // F(4,3): rows [4,0,-5,0,1,0] [0,-4,-4,1,1,0] [0,4,-4,-1,1,0] [0,-2,-1,2,1,0]
 //              [0,2,-1,-2,1,0] [0,4,0,-5,0,1]
 __device__ __forceinline__ void bt_1d(const float (&d)[6], float (&r)[6])
@@ -78,6 +87,14 @@ __device__ __forceinline__ void bt_1d(const float (&d)[8], float (&r)[8])
 // The same two transforms on two columns at once (packed f32x2 arithmetic: one
 // instruction per pair, each component rounded as in the scalar form).
 __device__ __forceinline__ float2 f2(float v) { return make_float2(v, v); }
+
+__device__ __forceinline__ void bt_1d(const float2 (&d)[4], float2 (&r)[4])
+{
+    r[0] = __ffma2_rn(f2(-1.f), d[2], d[0]);
+    r[1] = __fadd2_rn(d[1], d[2]);
+    r[2] = __ffma2_rn(f2(-1.f), d[1], d[2]);
+    r[3] = __ffma2_rn(f2(-1.f), d[3], d[1]);
+}
 
 __device__ __forceinline__ void bt_1d(const float2 (&d)[6], float2 (&r)[6])
 {
@@ -743,6 +760,8 @@ long long k1_by_gs(K1Op op, int gs, const wfq_plan *plan, const void *x, cudaStr
 long long k1_op(K1Op op, int m, bool f16, int gs, const wfq_plan *plan, const void *x, cudaStream_t s,
                 size_t smem)
 {
+    if (m == 2)
+        return f16 ? k1_by_gs<2, __half>(op, gs, plan, x, s, smem) : k1_by_gs<2, float>(op, gs, plan, x, s, smem);
     if (m == 4)
         return f16 ? k1_by_gs<4, __half>(op, gs, plan, x, s, smem) : k1_by_gs<4, float>(op, gs, plan, x, s, smem);
     return f16 ? k1_by_gs<6, __half>(op, gs, plan, x, s, smem) : k1_by_gs<6, float>(op, gs, plan, x, s, smem);
@@ -850,7 +869,7 @@ void plan_input_transform(wfq_plan &plan)
 cudaError_t setup_input_transform()
 {
     const int sizes[5] = {32, 64, 128, 256, 96};
-    for (int m = 4; m <= 6; m += 2)
+    for (int m = 2; m <= 6; m += 2)
         for (int f16 = 0; f16 < 2; ++f16)
             for (int gs : sizes) {
                 cudaError_t e = (cudaError_t)k1_op(kK1Setup, m, f16 != 0, gs, nullptr, nullptr, nullptr, 0);

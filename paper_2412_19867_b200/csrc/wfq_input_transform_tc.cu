@@ -686,7 +686,7 @@ void plan_input_transform_tc(wfq_plan &plan)
     K1TcPlan &k = plan.k1tc;
     const Geometry &g = plan.geo;
     k.use = false;
-    if (plan.in_dtype != WFQ_F16 || (g.gs != 32 && g.gs != 64) || g.C % TC_CB != 0) return;
+    if (plan.in_dtype != WFQ_F16 || (g.gs != 32 && g.gs != 64) || g.C % TC_CB != 0 || (g.m != 4 && g.m != 6)) return;
     if (plan.sm_count <= 0) return;
     const int n = g.n, m = g.m;
     const long long hw = (long long)g.H * g.W;

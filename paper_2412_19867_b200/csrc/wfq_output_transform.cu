@@ -11,6 +11,14 @@
 namespace wfq {
 namespace {
 
+// F(2,3), points 0, 1, -1, inf: V_A = [1,1,1,0; 0,1,-1,1] (the sign of the textbook's last column is
+// in the standard S_A).
+__device__ __forceinline__ void at_f23(const float (&v)[4], float (&o)[2])
+{
+    o[0] = v[0] + v[1] + v[2];
+    o[1] = v[1] - v[2] + v[3];
+}
+
 // 1-D output transform with V_A = V_{n x m}^T for the points 0, 1, -1, 2, -2, inf:
 //   o_u = sum_i f_i^u y_i (i < 5) + [u == 3] y_5
 __device__ __forceinline__ void at_f43(const float (&v)[6], float (&o)[4])
@@ -40,7 +48,9 @@ __device__ __forceinline__ void at_f63(const float (&v)[8], float (&o)[6])
 template <int M>
 __device__ __forceinline__ void at_1d(const float (&v)[M + 2], float (&o)[M])
 {
-    if constexpr (M == 4) at_f43(v, o); else at_f63(v, o);
+    if constexpr (M == 2) at_f23(v, o);
+    else if constexpr (M == 4) at_f43(v, o);
+    else at_f63(v, o);
 }
 
 // Optional epilogue on the spatial-domain outputs of one row segment: per-output-channel
@@ -240,7 +250,11 @@ cudaError_t launch_variant(const cudaLaunchConfig_t &cfg, const wfq_plan &plan, 
 // 10-19 KB of shared memory per SM.
 cudaError_t setup_output_transform()
 {
-    cudaError_t e = carveout<4, 1, false>();
+    cudaError_t e = carveout<2, 1, false>();
+    if (e == cudaSuccess) e = carveout<2, 0, false>();
+    if (e == cudaSuccess) e = carveout<2, 1, true>();
+    if (e == cudaSuccess) e = carveout<2, 0, true>();
+    if (e == cudaSuccess) e = carveout<4, 1, false>();
     if (e == cudaSuccess) e = carveout<6, 1, false>();
     if (e == cudaSuccess) e = carveout<4, 0, false>();
     if (e == cudaSuccess) e = carveout<6, 0, false>();
@@ -265,6 +279,10 @@ cudaError_t launch_output_transform(const wfq_plan &plan, float *y_dev, cudaStre
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     // y_dev is 16-byte aligned; rows of an even W keep 8-byte alignment for every tile
+    if (g.m == 2) {
+        if (g.W % 2 == 0) return launch_variant<2, 1>(cfg, plan, y_dev);
+        return launch_variant<2, 0>(cfg, plan, y_dev);
+    }
     if (g.m == 4) {
         if (g.W % 4 == 0) return launch_variant<4, 2>(cfg, plan, y_dev);
         if (g.W % 2 == 0) return launch_variant<4, 1>(cfg, plan, y_dev);

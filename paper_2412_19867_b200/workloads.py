@@ -25,9 +25,11 @@ BASE_SEED = 241219867
 
 # Standard F(m,3) scale vectors as printed in the paper's supplementary section
 # "Standard Winograd transforms" (input data for both sides, like the learned table).
-STD_SB = {4: [4.0, -6.0, -6.0, 24.0, 24.0, 1.0],
+STD_SB = {2: [1.0, 2.0, 2.0, -1.0],
+          4: [4.0, -6.0, -6.0, 24.0, 24.0, 1.0],
           6: [1.0, -4.5, -4.5, 90.0, 90.0, 45.0 / 32.0, 45.0 / 32.0, 1.0]}
-STD_SG = {4: [1.0 / 4, -1.0 / 6, -1.0 / 6, 1.0 / 24, 1.0 / 24, 1.0],
+STD_SG = {2: [1.0, 0.5, 0.5, 1.0],
+          4: [1.0 / 4, -1.0 / 6, -1.0 / 6, 1.0 / 24, 1.0 / 24, 1.0],
           6: [1.0, -2.0 / 9, -2.0 / 9, 1.0 / 90, 1.0 / 90, 32.0 / 45, 32.0 / 45, 1.0]}
 
 # Learned F(6,3) scales, table "Comparison between standard Winograd scales and our

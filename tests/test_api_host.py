@@ -44,7 +44,8 @@ def test_plan_create_validation(lib):
         (0, 64, 64, 32, 32, 4, 3, 32, 8): b.WFQ_ERR_INVALID_ARG,    # N < 1
         (1, 64, 64, -1, 32, 4, 3, 32, 8): b.WFQ_ERR_INVALID_ARG,    # H < 1
         (1, 64, 64, 32, 32, 4, 5, 32, 8): b.WFQ_ERR_UNSUPPORTED,    # r != 3
-        (1, 64, 64, 32, 32, 2, 3, 32, 8): b.WFQ_ERR_UNSUPPORTED,    # m not in {4,6}
+        (1, 64, 64, 32, 32, 3, 3, 32, 8): b.WFQ_ERR_UNSUPPORTED,    # m not in {2,4,6}
+        (1, 64, 64, 32, 32, 8, 3, 32, 8): b.WFQ_ERR_UNSUPPORTED,
         (1, 64, 64, 32, 32, 4, 3, 32, 4): b.WFQ_ERR_UNSUPPORTED,    # bits != 8
         (1, 64, 64, 32, 32, 4, 3, 48, 8): b.WFQ_ERR_UNSUPPORTED,    # group not multiple of 32
         (1, 96, 64, 32, 32, 4, 3, 64, 8): b.WFQ_ERR_UNSUPPORTED,    # C % group != 0

@@ -20,6 +20,7 @@ LAYERS = [
     Layer(1, 64, 48, 13, 11, 6, 64, "f16", "silu_outlier", "kaiming_chan", 8, 1, 0),     # ragged edges
     Layer(1, 128, 32, 8, 8, 4, 128, "f32", "gauss_outlier", "gauss_chan", 8, 2, 0),
     Layer(1, 256, 16, 12, 6, 6, 256, "f16", "silu_outlier", "kaiming", 8, 3, 0),
+    Layer(2, 64, 24, 7, 10, 2, 32, "f16", "silu_outlier", "kaiming_chan", 8, 4, 0),       # F(2,3)
 ]
 MODES = [("tile", 1), ("row", 2)]
 

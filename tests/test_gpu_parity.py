@@ -67,6 +67,11 @@ SMALL = [
     # groups of 256 (four lanes per group) and of 96 (group read twice from shared memory)
     Layer(1, 512, 32, 16, 16, 6, 256, "f16", "silu_outlier", "kaiming_chan", 5, 9, 1),
     Layer(2, 192, 32, 12, 24, 4, 96, "f16", "silu_outlier", "kaiming_chan", 5, 9, 2),
+    # F(2,3) (the textbook tile, 16 positions): even and odd widths, fp16 and fp32, 16-byte staging,
+    # both orientations of the contraction
+    Layer(2, 64, 96, 18, 24, 2, 64, "f16", "silu_outlier", "kaiming_chan", 5, 9, 3),
+    Layer(1, 128, 40, 9, 11, 2, 32, "f32", "gauss_outlier", "gauss_chan", 5, 9, 4),
+    Layer(1, 128, 256, 8, 6, 2, 128, "f16", "relu_heavy", "kaiming", 5, 9, 5),
 ]
 
 
@@ -111,8 +116,8 @@ def test_negative_and_standard_scales():
     _check(L, (x, w, np.array(learned["SB"], np.float32), np.array(learned["SG"], np.float32)))
 
 
-@pytest.mark.parametrize("m,H,W", [(4, 16, 16), (4, 9, 14), (4, 7, 7), (6, 12, 12), (6, 13, 11)],
-                         ids=["f43_w16", "f43_w14", "f43_w7", "f63_w12", "f63_w11"])
+@pytest.mark.parametrize("m,H,W", [(4, 16, 16), (4, 9, 14), (4, 7, 7), (6, 12, 12), (6, 13, 11), (2, 8, 10), (2, 7, 9)],
+                         ids=["f43_w16", "f43_w14", "f43_w7", "f63_w12", "f63_w11", "f23_w10", "f23_w9"])
 def test_bias_and_activation_epilogue(m, H, W):
     """y = act(conv + bias) fused into the output transform, every store variant; the
     setting can be changed and cleared between calls on one plan."""
@@ -146,8 +151,8 @@ def test_bias_and_activation_epilogue(m, H, W):
     conv.close()
 
 
-@pytest.mark.parametrize("m,H,W", [(4, 16, 16), (4, 9, 14), (4, 7, 7), (6, 12, 12), (6, 13, 11)],
-                         ids=["f43_w16", "f43_w14", "f43_w7", "f63_w12", "f63_w11"])
+@pytest.mark.parametrize("m,H,W", [(4, 16, 16), (4, 9, 14), (4, 7, 7), (6, 12, 12), (6, 13, 11), (2, 8, 10), (2, 7, 9)],
+                         ids=["f43_w16", "f43_w14", "f43_w7", "f63_w12", "f63_w11", "f23_w10", "f23_w9"])
 def test_fp16_output(m, H, W):
     """y written as fp16 by every store variant equals the fp32 result rounded once, with and
     without an epilogue, through the device and the host-buffer entry points, and in the
@@ -214,6 +219,7 @@ def test_contraction_shapes_agree(layer):
     Layer(1, 192, 32, 12, 24, 4, 96, "f16", "silu_outlier", "kaiming_chan", 9, 8, 4),     # generic group size
     Layer(2, 128, 48, 56, 56, 6, 64, "f16", "relu_heavy", "kaiming", 9, 8, 5),            # several items per CTA
     Layer(1, 512, 32, 16, 16, 4, 256, "f16", "silu_outlier", "kaiming_chan", 9, 8, 6),    # four lanes per group
+    Layer(2, 64, 32, 10, 14, 2, 64, "f16", "silu_outlier", "kaiming_chan", 9, 8, 7),      # F(2,3)
 ], ids=lambda L: L.name)
 def test_nhwc_input_matches_nchw(layer):
     """x given as [N][H][W][C] (TMA-staged input transform): codes and scales of stage 1 and the

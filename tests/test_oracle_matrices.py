@@ -47,7 +47,17 @@ def test_rebuilt_matrices_equal_printed(m, fixture):
     assert len(VB) == n and len(VA) == m and len(VG) == n
 
 
-@pytest.mark.parametrize("m", [4, 6])
+def test_f23_matrices_equal_the_textbook_ones():
+    """F(2,3) is not printed in the paper: the rebuilt matrices are pinned to the textbook ones."""
+    mats, errata = read_printed("winograd_f23_textbook.txt")
+    assert not errata
+    std = wm.STANDARD_SCALES[2]
+    assert std["SA"] == mats["SA"][0] and std["SB"] == mats["SB"][0] and std["SG"] == mats["SG"][0]
+    AT, BT, G = wm.scaled_matrices(2)
+    assert AT == mats["AT"] and BT == mats["BT"] and G == mats["G"]
+
+
+@pytest.mark.parametrize("m", [2, 4, 6])
 def test_scaling_condition_standard(m):
     std = wm.STANDARD_SCALES[m]
     assert all(a * b * g == 1 for a, b, g in zip(std["SA"], std["SB"], std["SG"]))
@@ -60,7 +70,7 @@ def _conv1d_via_winograd(AT, BT, G, d, g):
     return [sum(AT[u][i] * had[i] for i in range(len(had))) for u in range(len(AT))]
 
 
-@pytest.mark.parametrize("m", [4, 6])
+@pytest.mark.parametrize("m", [2, 4, 6])
 @pytest.mark.parametrize("scales", ["standard", "custom"])
 def test_minimal_filtering_identity_exact(m, scales):
     """A^T[(G g) .* (B^T d)] == sum_k d[u+k] g[k] for every pair of basis vectors."""
@@ -81,7 +91,7 @@ def test_minimal_filtering_identity_exact(m, scales):
 
 
 def test_inverse_is_exact():
-    for m in (4, 6):
+    for m in (2, 4, 6):
         V = wm.vandermonde(wm.POINTS[m], m + 2)
         I = wm.matmul(V, wm.inverse(V))
         assert all(I[i][j] == int(i == j) for i in range(m + 2) for j in range(m + 2))

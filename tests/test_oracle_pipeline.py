@@ -51,7 +51,7 @@ def test_direct_single_tap_shifts():
             np.testing.assert_array_equal(y, xp[a:a + 6, b:b + 5])
 
 
-@pytest.mark.parametrize("m", [4, 6])
+@pytest.mark.parametrize("m", [2, 4, 6])
 @pytest.mark.parametrize("shape", [(1, 2, 3, 7, 7), (2, 3, 2, 14, 9), (1, 1, 1, 4, 6), (1, 2, 2, 13, 56)])
 def test_unquantized_winograd_equals_direct(m, shape):
     rng = np.random.default_rng(3)
@@ -61,7 +61,7 @@ def test_unquantized_winograd_equals_direct(m, shape):
     assert np.max(np.abs(y - ref)) <= 1e-10 * np.max(np.abs(ref))
 
 
-@pytest.mark.parametrize("m", [4, 6])
+@pytest.mark.parametrize("m", [2, 4, 6])
 def test_scaling_invariance_unquantized(m):
     """Any nonzero S_B, S_G with S_A = (S_B S_G)^-1 give the same result."""
     rng = np.random.default_rng(4)
@@ -151,7 +151,7 @@ def test_dequantize_closed_form():
                 assert Y[p, t, k] == pytest.approx(want, rel=1e-15)
 
 
-@pytest.mark.parametrize("m", [4, 6])
+@pytest.mark.parametrize("m", [2, 4, 6])
 def test_one_channel_per_group_equals_direct(m):
     """With a single nonzero channel per group every nonzero maps to +-127 and
     dequantizes to 127*fl32(amax/127): the quantized pipeline must reproduce the direct
@@ -199,7 +199,7 @@ def test_quantized_error_within_a_priori_bound(m, gs):
     assert orc.sqnr_db(ref, res.y) > 15.0
 
 
-@pytest.mark.parametrize("m", [4, 6])
+@pytest.mark.parametrize("m", [2, 4, 6])
 def test_codes_invariant_to_scales_up_to_sign(m):
     """Groups run along channels at a fixed position, so multiplying a position by
     sB_i sB_j scales the whole group: codes change only by the sign of that product."""
