@@ -9,8 +9,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwfq.so")
 SOURCES = ["wfq_api.cu", "wfq_filter_prep.cu", "wfq_input_transform.cu", "wfq_input_transform_tc.cu",
-           "wfq_gemm.cu", "wfq_output_transform.cu", "wfq_full_quant.cu"]
-HEADERS = ["wfq_internal.h", "wfq_ptx.cuh"]
+           "wfq_input_transform_tcn.cu", "wfq_gemm.cu", "wfq_output_transform.cu", "wfq_full_quant.cu"]
+HEADERS = ["wfq_internal.h", "wfq_ptx.cuh", "wfq_quant.cuh"]
 
 
 def _nvcc():

@@ -62,7 +62,7 @@ wfq_status_t bind_device(wfq_plan *plan)
         if (!g_device_ready[dev]) {
             if (wfq::setup_input_transform() != cudaSuccess || wfq::setup_input_transform_tc() != cudaSuccess ||
                 wfq::setup_gemm() != cudaSuccess || wfq::setup_output_transform() != cudaSuccess ||
-                wfq::setup_full_quant() != cudaSuccess)
+                wfq::setup_full_quant() != cudaSuccess || wfq::setup_input_transform_tcn() != cudaSuccess)
                 return WFQ_ERR_CUDA;
             g_device_ready[dev] = true;
         }
@@ -199,8 +199,13 @@ wfq_status_t wfq_plan_set_input_layout(wfq_plan_t *plan, wfq_layout_t layout)
     if (layout == WFQ_NHWC && plan->fq_input) return WFQ_ERR_UNSUPPORTED;   // integer input transform: NCHW only
     plan->in_nhwc = layout == WFQ_NHWC;
     plan->tmap_xn_base = nullptr;
+    plan->tmap_xn_tc_base = nullptr;
     for (int i = 0; i < 2; ++i)
-        if (plan->sub[i]) { plan->sub[i]->in_nhwc = plan->in_nhwc; plan->sub[i]->tmap_xn_base = nullptr; }
+        if (plan->sub[i]) {
+            plan->sub[i]->in_nhwc = plan->in_nhwc;
+            plan->sub[i]->tmap_xn_base = nullptr;
+            plan->sub[i]->tmap_xn_tc_base = nullptr;
+        }
     return WFQ_OK;
 }
 

@@ -864,6 +864,7 @@ void plan_input_transform(wfq_plan &plan)
     if (plan.in_dtype == WFQ_F16 && plan.geo.W % 8 == 0) plan_k1(plan, plan.k1v, true);
     plan_k1_nhwc(plan);
     plan.tmap_xn_base = nullptr;
+    plan.tmap_xn_tc_base = nullptr;
 }
 
 cudaError_t setup_input_transform()
@@ -886,6 +887,25 @@ cudaError_t launch_input_transform(wfq_plan &plan, const void *x_dev, cudaStream
     if (plan.in_nhwc) {
         // x[N][H][W][C] as a 4-D tensor (C, W, H, N) with boxes of one work item's strip
         if ((reinterpret_cast<uintptr_t>(x_dev) & 15u) != 0) return cudaErrorInvalidValue;
+        const unsigned long long esz0 = plan.in_dtype == WFQ_F16 ? 2 : 4;
+        // tensor cores where they apply (fp16, groups of 32 or 64, C a multiple of 64, F(4,3) / F(6,3)),
+        // unless the debug option asks for the plain kernel
+        if (input_transform_tcn_applies(plan) && plan.k1_choice != 1) {
+            if (plan.tmap_xn_tc_base != x_dev) {
+                const unsigned long long dims[4] = {(unsigned long long)g.C, (unsigned long long)g.W,
+                                                    (unsigned long long)g.H, (unsigned long long)g.N};
+                const unsigned long long strides[3] = {(unsigned long long)g.C * esz0,
+                                                       (unsigned long long)g.W * g.C * esz0,
+                                                       (unsigned long long)g.H * g.W * g.C * esz0};
+                unsigned box[4];
+                input_transform_tcn_box(plan, box);
+                if (!encode_tmap(&plan.tmap_xn_tc, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, x_dev, dims, strides, box,
+                                 CU_TENSOR_MAP_SWIZZLE_128B))
+                    return cudaErrorInvalidValue;
+                plan.tmap_xn_tc_base = x_dev;
+            }
+            return launch_input_transform_tcn(plan, stream);
+        }
         if (plan.tmap_xn_base != x_dev) {
             const unsigned long long esz = plan.in_dtype == WFQ_F16 ? 2 : 4;
             const unsigned long long dims[4] = {(unsigned long long)g.C, (unsigned long long)g.W,

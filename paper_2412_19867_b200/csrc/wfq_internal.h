@@ -126,6 +126,8 @@ struct wfq_plan {
     bool in_nhwc = false;      // x is [N][H][W][C] instead of [N][C][H][W]
     CUtensorMap tmap_xn;       // the NHWC input as (C, W, H, N)
     const void *tmap_xn_base = nullptr;   // x pointer tmap_xn was encoded for
+    CUtensorMap tmap_xn_tc;    // the same with the boxes of the tensor-core NHWC input transform
+    const void *tmap_xn_tc_base = nullptr;
     wfq::K1TcPlan k1tc;
     CUtensorMap tmap_x;        // the input tensor as the tensor-core input transform stages it
     const void *tmap_x_base = nullptr;   // x pointer tmap_x was encoded for
@@ -164,6 +166,10 @@ cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *
                                cudaStream_t stream);
 cudaError_t launch_input_transform(wfq_plan &plan, const void *x_dev, cudaStream_t stream);
 cudaError_t launch_input_transform_tc(const wfq_plan &plan, const void *x_dev, cudaStream_t stream);
+bool input_transform_tcn_applies(const wfq_plan &plan);
+void input_transform_tcn_box(const wfq_plan &plan, unsigned (&box)[4]);
+cudaError_t setup_input_transform_tcn();
+cudaError_t launch_input_transform_tcn(const wfq_plan &plan, cudaStream_t stream);
 
 // Per-plan launch parameters (host only, no device work) and per-device one-time kernel
 // attributes (shared-memory sizes and carveouts).
