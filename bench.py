@@ -74,6 +74,9 @@ def parse_args():
     ap.add_argument("--k1-kernel", type=int, default=0, choices=[0, 1, 2],
                     help="input-transform kernel: 0 the library's choice, 1 cp.async, 2 tensor cores "
                          "where they apply (profiling)")
+    ap.add_argument("--nhwc", action="store_true",
+                    help="hand x over as [N][H][W][C] (the library then uses its NHWC input transforms); the "
+                         "default workload is NCHW")
     ap.add_argument("--cpu-seconds", type=float, default=16.0,
                     help="CPU time budget of the oracle baseline")
     return ap.parse_args()
@@ -528,7 +531,7 @@ def run_wfq(args):
         torch.cuda.synchronize(dev)
 
     wk = Workload(args.config, args.only_layer, dev, stream, flush, use_graph=not args.no_graph,
-                  k1_kernel=args.k1_kernel)
+                  k1_kernel=args.k1_kernel, nhwc=args.nhwc)
     for _ in range(warmup):
         flush.zero_()
         wk.step()

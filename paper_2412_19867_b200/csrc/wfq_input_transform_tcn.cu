@@ -10,8 +10,11 @@
 // along the row, 128-byte swizzle), which is an MN-major B operand of tcgen05.mma kind::f16 with
 // K = the patch elements (8 per patch row: for F(4,3) the two extra columns meet zero columns of the
 // matrix) and N = the 64 channels.  Accumulator rows (TMEM lanes) = (tile of the work item, Winograd
-// position): the A operand is the block-diagonal matrix [tile][position] x [tile][patch element],
-// K-major in shared memory, copied once per CTA from a global image the host builds.  A quantizer
+// position), PL rows per tile: the A operand of tile t's MMAs is the constant matrix [position] x
+// [patch element] with its rows at t * PL and zeros elsewhere.  Shared memory holds the matrix once,
+// K-major, between (TB - 1) * PL zero rows and 128 - PL zero rows, and tile t's descriptor starts
+// t * PL rows before the matrix (PL is a multiple of 8, so the 128-byte swizzle keeps its phase);
+// only the matrix itself (5-8 KB) is copied from a global image the host builds.  A quantizer
 // thread then owns one (tile, position) and reads its 64 channels with tcgen05.ld: abs-max over
 // registers, scale, 64 contiguous codes; no im2col, no fp32 round trip through shared memory.
 //
@@ -46,12 +49,14 @@ template <int M>
 struct TnCfg {
     static constexpr int NN = M + 2;
     static constexpr int P = NN * NN;
-    static constexpr int TB = M == 6 ? 2 : 3;                 // tiles per work item: TB * P <= 128 rows
-    static constexpr int KT = NN * 8;                         // K elements per tile (8 columns per patch row)
+    static constexpr int TB = M == 6 ? 2 : 3;                 // tiles per work item
+    static constexpr int PL = M == 6 ? 64 : 40;               // accumulator rows per tile (>= P, a multiple of 8)
+    static constexpr int KT = NN * 8;                         // K elements per tile (8 columns per patch row), <= 64
     static constexpr int KSTEPS = KT / 16;                    // MMAs per tile
-    static constexpr int KTOT = TB * KT;                      // 128 or 144
-    static constexpr int KBLK = (KTOT + 63) / 64;             // 64-element blocks of the A operand
-    static constexpr int A_BYTES = KBLK * 128 * 128;          // [KBLK][128 rows][128 B], swizzled
+    static constexpr int Z0 = (TB - 1) * PL;                  // zero rows before the matrix
+    static constexpr int A_ROWS = Z0 + 128;                   // zero rows, matrix, zero rows
+    static constexpr int A_BYTES = (A_ROWS * 128 + 1023) / 1024 * 1024;   // rows of 64 fp16, 128-byte swizzle
+    static constexpr int AMAT_BYTES = PL * 128;               // the matrix itself
     static constexpr int BOX_BYTES = NN * 8 * 128;            // one tile's box
     static constexpr int STRIP_BYTES = TB * BOX_BYTES;
     static constexpr size_t SMEM_BYTES = 1024 + A_BYTES + TN_NSTRIP * STRIP_BYTES;
@@ -71,7 +76,7 @@ struct TnArgs {
     float *sX;
     int *status;
     long long wait_cycles;
-    const uint4 *amat;        // the A operand as it lies in shared memory, A_BYTES
+    const uint4 *amat;        // the constant matrix as it lies in shared memory, AMAT_BYTES
     int NCH, NCB, items;      // chunks of TB tiles per tile row, channel blocks, work items
     int debug_skip_item;      // >= 0: the producer skips this item's copies (exercises the bounded waits)
 };
@@ -108,9 +113,13 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
         ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TN_TMEM_COLS);
         ptx::tmem_relinquish();
     }
-    // the constant matrix: a plain copy (it does not depend on the previous kernel)
-    for (int i = threadIdx.x; i < C::A_BYTES / 16; i += TN_THREADS)
-        reinterpret_cast<uint4 *>(amat_s)[i] = __ldg(a.amat + i);
+    // the A operand: zero rows, the constant matrix (a plain copy; it does not depend on the previous
+    // kernel), zero rows
+    for (int i = threadIdx.x; i < C::A_BYTES / 16; i += TN_THREADS) {
+        const int j = i - C::Z0 * 8;                           // 16-byte pieces: 8 per row
+        reinterpret_cast<uint4 *>(amat_s)[i] =
+            (j >= 0 && j < C::AMAT_BYTES / 16) ? __ldg(a.amat + j) : make_uint4(0u, 0u, 0u, 0u);
+    }
     ptx::fence_proxy_async_smem();      // the tensor cores read it through the async proxy
     ptx::tc_fence_before();
     __syncthreads();
@@ -175,8 +184,8 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
                 for (int tl = 0; tl < C::TB; ++tl)
 #pragma unroll
                     for (int ks = 0; ks < C::KSTEPS; ++ks) {
-                        const int koff = tl * C::KT + ks * 16;                  // first K element of this MMA
-                        const uint32_t al = a_lo0 + (uint32_t)((koff / 64) * (128 * 128 / 16) + (koff % 64) / 8);
+                        // the matrix's rows land on accumulator rows tl * PL ...: start tl * PL rows early
+                        const uint32_t al = a_lo0 + (uint32_t)(((C::Z0 - tl * C::PL) * 128 + ks * 32) >> 4);
                         const uint32_t bl = b_lo + (uint32_t)((tl * C::BOX_BYTES + ks * 2048) >> 4);
                         if (tl == 0 && ks == 0) ptx::umma_f16_lo<false>(d, al, bl, dhi, idesc);
                         else ptx::umma_f16_lo<true>(d, al, bl, dhi, idesc);
@@ -192,8 +201,8 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
         // ---------------- quantizers ----------------
         const int quarter = warp & 3;
         const int r = quarter * 32 + lane;                    // accumulator row = tile * P + position
-        const int tl = r / C::P, p = r - tl * C::P;
-        const bool row_ok = r < C::TB * C::P;
+        const int tl = r / C::PL, p = r - tl * C::PL;
+        const bool row_ok = tl < C::TB && p < C::P;
         const float sp = row_ok ? tab.in_scale[p] : 0.f, sl = row_ok ? tab.in_scale_lo[p] : 0.f;
         const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16);
         int slot = 0;
@@ -269,29 +278,27 @@ const float kTnBT6[64] = {
     0, -0.5f, 0.25f, 2.5f, -1.25f, -2, 1, 0, 0, 2, 4, -2.5f, -5, 0.5f, 1, 0,
     0, -2, 4, 2.5f, -5, -0.5f, 1, 0,         0, -1, 0, 5.25f, 0, -5.25f, 0, 1};
 
-// The A operand as it lies in shared memory: [KBLK][128 rows][64 fp16], K-major with the 128-byte
-// swizzle (16-byte chunk c of row r is stored at chunk c ^ (r & 7)).  Row tl * P + (i, j), K element
-// tl * KT + a * 8 + b holds BT[i][a] * BT[j][b] (b < n), everything else is zero.
+// The constant matrix as it lies in shared memory: [PL rows][64 fp16], K-major with the 128-byte
+// swizzle (16-byte chunk c of row r is stored at chunk c ^ (r & 7); the matrix starts at a multiple of
+// 8 rows).  Row (i, j), K element a * 8 + b holds BT[i][a] * BT[j][b] (b < n); everything else is zero.
 template <int M>
 void build_amat(std::vector<uint16_t> &out)
 {
     using C = TnCfg<M>;
     const float *bt = M == 6 ? kTnBT6 : kTnBT4;
-    out.assign((size_t)C::A_BYTES / 2, 0);
-    for (int tl = 0; tl < C::TB; ++tl)
-        for (int p = 0; p < C::P; ++p) {
-            const int i = p / C::NN, j = p % C::NN, r = tl * C::P + p;
-            for (int aa = 0; aa < C::NN; ++aa)
-                for (int b = 0; b < C::NN; ++b) {
-                    const int k = tl * C::KT + aa * 8 + b;
-                    const int kb = k / 64, kk = k % 64;
-                    const int chunk = (kk / 8) ^ (r & 7);
-                    const __half h = __float2half_rn(bt[i * C::NN + aa] * bt[j * C::NN + b]);
-                    uint16_t bits;
-                    memcpy(&bits, &h, 2);
-                    out[((size_t)kb * 128 + r) * 64 + chunk * 8 + (kk % 8)] = bits;
-                }
-        }
+    out.assign((size_t)C::AMAT_BYTES / 2, 0);
+    for (int p = 0; p < C::P; ++p) {
+        const int i = p / C::NN, j = p % C::NN;
+        for (int aa = 0; aa < C::NN; ++aa)
+            for (int b = 0; b < C::NN; ++b) {
+                const int k = aa * 8 + b;
+                const int chunk = (k / 8) ^ (p & 7);
+                const __half h = __float2half_rn(bt[i * C::NN + aa] * bt[j * C::NN + b]);
+                uint16_t bits;
+                memcpy(&bits, &h, 2);
+                out[(size_t)p * 64 + chunk * 8 + (k % 8)] = bits;
+            }
+    }
 }
 
 constexpr int kTnMaxDevices = 64;
