@@ -808,10 +808,14 @@ def run_wfq(args):
             torch.cuda.synchronize(dev)
             ms = [statistics.median(w4.timed_replays(reps)) for _ in range(10)]
             s4, _, _ = w4.summary(statistics.mean(ms), w4.kernel_split(10), peak)
-            same = all(torch.equal(a, b_) for a, b_ in zip(w4.ys, ys_headline))
+            # the tensor-core transform rounds V in another order than the NCHW kernel: a code in about
+            # 1e-6 may differ by one step, so the outputs are compared in norm, not bit for bit
+            dev_rel = max(float(torch.linalg.vector_norm(a.float() - b_.float()) /
+                                torch.linalg.vector_norm(b_.float())) for a, b_ in zip(w4.ys, ys_headline))
             nhwc = {"workload": s4["workload"], "value": s4["value"], "unit": UNIT, "us_per_step": s4["us_per_step"],
                     "input_transform_us_per_step": s4["kernels"][KERNELS[0]]["us_per_step"],
-                    "equals_nchw_result": bool(same)}
+                    "kernel": "input_transform_tcn_kernel (TMA box as the MN-major operand of tcgen05.mma kind::f16)",
+                    "rel_l2_vs_nchw_result": dev_rel, "agrees_with_nchw_result": bool(dev_rel <= 1e-4)}
             w4.close()
             del w4
             torch.cuda.empty_cache()

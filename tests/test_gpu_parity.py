@@ -419,6 +419,7 @@ def test_bounded_waits_run_out_and_report():
     # (the roles up- and downstream of the starved one run out at about the same time: any of the
     # kernel's waits may be the first to record itself)
     cases = [(b.WFQ_DEBUG_SKIP_INPUT_ITEM, 1, "k1", set(range(8, 14))),   # tensor-core input transform
+             (b.WFQ_DEBUG_SKIP_INPUT_ITEM, 1, "k1n", set(range(8, 14))),  # the same for NHWC input
              (b.WFQ_DEBUG_SKIP_GEMM_STAGE, 0, "k2", set(range(1, 8)))]    # contraction
     for option, value, stage, want in cases:
         conv, (x, w, sB, sG) = make_conv(L)
@@ -427,10 +428,14 @@ def test_bounded_waits_run_out_and_report():
         torch.cuda.synchronize()
         conv.check_status()
         b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_WAIT_CYCLES, 2_000_000)   # about 1 ms
-        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, 2)
+        b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, 0 if stage == "k1n" else 2)
         b.wfq_plan_set_debug_option(conv.plan, option, value)
         if stage == "k1":
             b.wfq_input_transform_quantize(conv.plan, xd.data_ptr(), conv._stream())
+        elif stage == "k1n":
+            conv.set_input_layout("nhwc")
+            xn = xd.permute(0, 2, 3, 1).contiguous()
+            b.wfq_input_transform_quantize(conv.plan, xn.data_ptr(), conv._stream())
         else:
             b.wfq_gemm_dequantize(conv.plan, conv._stream())
         torch.cuda.synchronize()                              # the kernel ended by itself
