@@ -149,6 +149,19 @@ wfq_status_t wfq_plan_set_input_layout(wfq_plan_t *plan, wfq_layout_t layout);
 wfq_status_t wfq_plan_set_output_dtype(wfq_plan_t *plan, wfq_dtype_t dtype);
 
 /*
+ * Bit width of the filter codes: 8 (default) or 4 (WFQ_ERR_UNSUPPORTED otherwise).  With 4 the
+ * offline filter path quantizes each channel group of the transformed filters to codes in
+ * [-7, 7] with scale = amax / 7 (the quantizer of the header comment with 7 in place of 127): the
+ * "W4A8" setting of the paper's experiments (Section 5), which the paper applies to its other
+ * layers and which is offered here for the Winograd layers as well.  Activations stay at 8 bits.
+ * On the device the codes remain one per byte, because the contraction is an int8 tensor-core
+ * product either way and is not bound by the filter stream; the exported blob stores two per
+ * byte.  Changing the width invalidates prepared filters: call wfq_prepare_filters (or
+ * wfq_filters_import) afterwards.  Host only.
+ */
+wfq_status_t wfq_plan_set_weight_bits(wfq_plan_t *plan, int bits);
+
+/*
  * The paper's fully quantized transforms (Section 4.1), off by default.
  *   quant_input  1: the input transform runs on integer codes (Eq. quant-B): x is quantized to 8
  *                bits with one scale per (tile, channel group) over the group's n x n patches,
@@ -260,14 +273,16 @@ wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev,
  * Prepared filters as a host blob, so that wfq_prepare_filters can run once, offline, and a later
  * process only loads its result (the filter path is offline in the paper as well, Section 4.1).
  * The blob holds a 256-byte header (layer shape, tile and group size, the three scale vectors in
- * fp64), Wq [P][K][C] int8 and sW [P][G][Kp] fp32; it is tied to those parameters, not to the
- * batch size or the image size.
+ * fp64, the weight bit width), Wq [P][K][C] and sW [P][G][Kp] fp32; it is tied to those parameters,
+ * not to the batch size or the image size.  Wq is one int8 code per byte for 8-bit weights and two
+ * codes per byte for 4-bit weights (byte j: code 2j in the low nibble, code 2j+1 in the high nibble,
+ * two's complement), which halves the blob.
  *   wfq_filters_bytes   size of the blob for this plan
  *   wfq_filters_export  host_buf (host, >= that size, caller-owned) receives the blob of a
  *                       prepared plan; synchronous with respect to `stream`
  *   wfq_filters_import  makes the plan prepared from a blob written for the same C, K, tile and
- *                       group size (WFQ_ERR_INVALID_ARG otherwise, plan unchanged); the blob is
- *                       copied before the call returns
+ *                       group size (WFQ_ERR_INVALID_ARG otherwise, plan unchanged); the plan takes
+ *                       the blob's weight bit width; the blob is copied before the call returns
  */
 size_t wfq_filters_bytes(const wfq_plan_t *plan);
 wfq_status_t wfq_filters_export(wfq_plan_t *plan, void *host_buf, size_t bytes, void *stream);

@@ -31,7 +31,7 @@ EXPORTS = [
     "wfq_output_transform", "wfq_debug_gemm_acc32", "wfq_debug_get",
     "wfq_check_device_status", "wfq_plan_destroy", "wfq_status_string", "wfq_version",
     "wfq_quantize_filters_static", "wfq_plan_set_debug_option", "wfq_debug_int8_mma_rate",
-    "wfq_plan_set_epilogue", "wfq_plan_set_full_quant", "wfq_plan_set_output_dtype",
+    "wfq_plan_set_epilogue", "wfq_plan_set_full_quant", "wfq_plan_set_output_dtype", "wfq_plan_set_weight_bits",
     "wfq_conv_forward_host_async", "wfq_filters_bytes", "wfq_filters_export", "wfq_filters_import",
     "wfq_plan_set_input_layout",
 ]
@@ -79,6 +79,7 @@ def load():
     lib.wfq_plan_set_epilogue.argtypes = [vp, vp, ci]
     lib.wfq_plan_set_full_quant.argtypes = [vp, ci, ci]
     lib.wfq_plan_set_output_dtype.argtypes = [vp, ci]
+    lib.wfq_plan_set_weight_bits.argtypes = [vp, ci]
     lib.wfq_plan_set_input_layout.argtypes = [vp, ci]
     lib.wfq_plan_set_debug_option.argtypes = [vp, ci, ctypes.c_longlong]
     lib.wfq_debug_int8_mma_rate.argtypes = [vp, ci, ci, ctypes.POINTER(ctypes.c_longlong), vp]
@@ -128,6 +129,10 @@ def wfq_plan_set_epilogue(plan, bias_dev, act=WFQ_ACT_NONE):
 
 def wfq_plan_set_input_layout(plan, layout):
     _check(load().wfq_plan_set_input_layout(plan, layout), "wfq_plan_set_input_layout")
+
+
+def wfq_plan_set_weight_bits(plan, bits):
+    _check(load().wfq_plan_set_weight_bits(plan, bits), "wfq_plan_set_weight_bits")
 
 
 def wfq_plan_set_output_dtype(plan, dtype):
@@ -283,6 +288,10 @@ class Conv:
         """"nchw" (default) or "nhwc": forward() then takes x of shape (N, H, W, C)."""
         self.in_layout = layout
         wfq_plan_set_input_layout(self.plan, WFQ_NHWC if layout == "nhwc" else WFQ_NCHW)
+
+    def set_weight_bits(self, bits):
+        """8 (default) or 4; call before prepare()."""
+        wfq_plan_set_weight_bits(self.plan, bits)
 
     def set_output_dtype(self, dtype):
         """"f32" (default) or "f16": element type of the tensors forward() returns or fills."""

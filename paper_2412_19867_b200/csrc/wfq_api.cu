@@ -233,6 +233,19 @@ wfq_status_t wfq_plan_set_output_dtype(wfq_plan_t *plan, wfq_dtype_t dtype)
     return WFQ_OK;
 }
 
+wfq_status_t wfq_plan_set_weight_bits(wfq_plan_t *plan, int bits)
+{
+    if (!plan) return WFQ_ERR_INVALID_ARG;
+    if (bits != 8 && bits != 4) return WFQ_ERR_UNSUPPORTED;
+    if (bits != plan->w_bits) {
+        plan->w_bits = bits;
+        plan->prepared = false;    // filters quantized at the other width are not valid any more
+        for (int i = 0; i < 2; ++i)
+            if (plan->sub[i]) plan->sub[i]->prepared = false;
+    }
+    return WFQ_OK;
+}
+
 wfq_status_t wfq_plan_set_full_quant(wfq_plan_t *plan, int quant_input, wfq_y_quant_t y_mode)
 {
     if (!plan) return WFQ_ERR_INVALID_ARG;
@@ -357,7 +370,7 @@ wfq_status_t wfq_prepare_filters(wfq_plan_t *plan, const float *w_dev, const flo
 namespace {
 struct FilterBlobHeader {
     char magic[8];                       // "WFQFILT1"
-    int32_t m, C, K, gs, P, G, Kp, reserved;
+    int32_t m, C, K, gs, P, G, Kp, w_bits;   // w_bits: 8, 4, or 0 (= 8, blobs written before the field existed)
     double sB[wfq::kMaxN], sG[wfq::kMaxN], sA[wfq::kMaxN];
     char pad[256 - 8 - 8 * 4 - 3 * 8 * wfq::kMaxN];
 };
@@ -365,11 +378,18 @@ static_assert(sizeof(FilterBlobHeader) == 256, "header is 256 bytes");
 const char kBlobMagic[8] = {'W', 'F', 'Q', 'F', 'I', 'L', 'T', '1'};
 }  // namespace
 
+// bytes of the code section: one code per byte, or two per byte for 4-bit weights
+static size_t blob_wq_bytes(const wfq::Geometry &g, int w_bits)
+{
+    const size_t codes = (size_t)g.P * g.K * g.C;
+    return w_bits == 4 ? codes / 2 : codes;
+}
+
 size_t wfq_filters_bytes(const wfq_plan_t *plan)
 {
     if (!plan) return 0;
     const wfq::Geometry &g = plan->geo;
-    return sizeof(FilterBlobHeader) + (size_t)g.P * g.K * g.C + (size_t)g.P * g.G * g.Kp * sizeof(float);
+    return sizeof(FilterBlobHeader) + blob_wq_bytes(g, plan->w_bits) + (size_t)g.P * g.G * g.Kp * sizeof(float);
 }
 
 wfq_status_t wfq_filters_export(wfq_plan_t *plan, void *host_buf, size_t bytes, void *stream)
@@ -381,15 +401,28 @@ wfq_status_t wfq_filters_export(wfq_plan_t *plan, void *host_buf, size_t bytes, 
     FilterBlobHeader h;
     memset(&h, 0, sizeof(h));
     memcpy(h.magic, kBlobMagic, 8);
-    h.m = g.m; h.C = g.C; h.K = g.K; h.gs = g.gs; h.P = g.P; h.G = g.G; h.Kp = g.Kp;
+    h.m = g.m; h.C = g.C; h.K = g.K; h.gs = g.gs; h.P = g.P; h.G = g.G; h.Kp = g.Kp; h.w_bits = plan->w_bits;
     for (int i = 0; i < g.n; ++i) { h.sB[i] = plan->sB[i]; h.sG[i] = plan->sG[i]; h.sA[i] = plan->sA[i]; }
     memcpy(host_buf, &h, sizeof(h));
     char *dst = static_cast<char *>(host_buf) + sizeof(h);
-    const size_t wq_bytes = (size_t)g.P * g.K * g.C, sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
+    const size_t codes = (size_t)g.P * g.K * g.C, wq_bytes = blob_wq_bytes(g, plan->w_bits);
+    const size_t sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
     cudaStream_t st = as_stream(stream);
-    if (cudaMemcpyAsync(dst, plan->Wq, wq_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaMemcpyAsync(dst + wq_bytes, plan->sW, sw_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return WFQ_ERR_CUDA;
+    void *packed = nullptr;
+    const void *src = plan->Wq;
+    if (plan->w_bits == 4) {
+        // two codes per byte, packed on the device into a stream-ordered temporary
+        if (cudaMallocAsync(&packed, wq_bytes, st) != cudaSuccess) return WFQ_ERR_CUDA;
+        if (wfq::launch_pack_nibbles(plan->Wq, packed, codes, st) != cudaSuccess) {
+            cudaFreeAsync(packed, st);
+            return WFQ_ERR_CUDA;
+        }
+        src = packed;
+    }
+    bool ok = cudaMemcpyAsync(dst, src, wq_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+              cudaMemcpyAsync(dst + wq_bytes, plan->sW, sw_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (packed) ok = (cudaFreeAsync(packed, st) == cudaSuccess) && ok;
+    if (!ok) return WFQ_ERR_CUDA;
     return cuda_status(cudaStreamSynchronize(st));
 }
 
@@ -400,8 +433,12 @@ wfq_status_t wfq_filters_import(wfq_plan_t *plan, const void *host_buf, size_t b
     FilterBlobHeader h;
     memcpy(&h, host_buf, sizeof(h));
     if (memcmp(h.magic, kBlobMagic, 8) != 0 || h.m != g.m || h.C != g.C || h.K != g.K || h.gs != g.gs ||
-        h.P != g.P || h.G != g.G || h.Kp != g.Kp || bytes < wfq_filters_bytes(plan))
+        h.P != g.P || h.G != g.G || h.Kp != g.Kp || (h.w_bits != 0 && h.w_bits != 8 && h.w_bits != 4))
         return WFQ_ERR_INVALID_ARG;
+    const int w_bits = h.w_bits == 4 ? 4 : 8;
+    const size_t codes = (size_t)g.P * g.K * g.C, wq_bytes = blob_wq_bytes(g, w_bits);
+    const size_t sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
+    if (bytes < sizeof(FilterBlobHeader) + wq_bytes + sw_bytes) return WFQ_ERR_INVALID_ARG;
     for (int i = 0; i < g.n; ++i)
         if (!std::isfinite(h.sB[i]) || !std::isfinite(h.sG[i]) || !std::isfinite(h.sA[i]) || h.sB[i] == 0.0 ||
             h.sG[i] == 0.0 || h.sA[i] == 0.0)
@@ -411,10 +448,18 @@ wfq_status_t wfq_filters_import(wfq_plan_t *plan, const void *host_buf, size_t b
     if (bs != WFQ_OK) return bs;
     for (int i = 0; i < g.n; ++i) { plan->sB[i] = h.sB[i]; plan->sG[i] = h.sG[i]; plan->sA[i] = h.sA[i]; }
     fill_scale_tables(plan);
+    plan->w_bits = w_bits;
     const char *src = static_cast<const char *>(host_buf) + sizeof(h);
-    const size_t wq_bytes = (size_t)g.P * g.K * g.C, sw_bytes = (size_t)g.P * g.G * g.Kp * sizeof(float);
-    if (cudaMemcpyAsync(plan->Wq, src, wq_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(plan->sW, src + wq_bytes, sw_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    if (w_bits == 4) {
+        void *packed = nullptr;
+        if (cudaMallocAsync(&packed, wq_bytes, st) != cudaSuccess) return WFQ_ERR_CUDA;
+        const bool ok = cudaMemcpyAsync(packed, src, wq_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                        wfq::launch_unpack_nibbles(packed, plan->Wq, codes, st) == cudaSuccess;
+        if (cudaFreeAsync(packed, st) != cudaSuccess || !ok) return WFQ_ERR_CUDA;
+    } else if (cudaMemcpyAsync(plan->Wq, src, wq_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        return WFQ_ERR_CUDA;
+    }
+    if (cudaMemcpyAsync(plan->sW, src + wq_bytes, sw_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return WFQ_ERR_CUDA;
     // the caller may free or change the blob when this returns
     if (cudaStreamSynchronize(st) != cudaSuccess) return WFQ_ERR_CUDA;

@@ -58,12 +58,14 @@ __global__ void filter_transform_kernel(const float *__restrict__ w, float *__re
         }
 }
 
-// One thread per (p, k, g): abs-max of the group, scale, codes.  sW rows are k_pitch
-// floats apart.
+// One thread per (p, k, g): abs-max of the group, scale, codes in [-qmax, qmax] (127 for 8-bit
+// weights, 7 for 4-bit weights; the codes are stored one per byte either way, which is what the
+// int8 tensor-core contraction reads).  sW rows are k_pitch floats apart.
 __global__ void filter_quantize_kernel(const float *__restrict__ w32, int8_t *__restrict__ Wq,
                                        float *__restrict__ sW, int P, int K, int C, int gs,
-                                       int k_pitch)
+                                       int k_pitch, int qmax)
 {
+    const float fq = (float)qmax;
     const int G = C / gs;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)P * K * G) return;
@@ -76,13 +78,13 @@ __global__ void filter_quantize_kernel(const float *__restrict__ w32, int8_t *__
     for (int e = 0; e < gs; ++e) amax = fmaxf(amax, fabsf(src[e]));
     float scale = 0.f, inv = 0.f;
     if (amax >= 1e-30f) {
-        scale = __fdiv_rn(amax, 127.f);
-        inv = __fdiv_rn(127.f, amax);
+        scale = __fdiv_rn(amax, fq);
+        inv = __fdiv_rn(fq, amax);
     }
     sW[((size_t)p * G + g) * k_pitch + k] = scale;
     for (int e = 0; e < gs; ++e) {
         int q = __float2int_rn(__fmul_rn(src[e], inv));
-        q = max(-127, min(127, q));
+        q = max(-qmax, min(qmax, q));
         dst[e] = (int8_t)q;
     }
 }
@@ -108,9 +110,63 @@ cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *
         const int threads = 128;
         const unsigned blocks = (unsigned)((total + threads - 1) / threads);
         filter_quantize_kernel<<<blocks, threads, 0, stream>>>(scratch_w32, plan.Wq, plan.sW, g.P,
-                                                               g.K, g.C, g.gs, g.Kp);
+                                                               g.K, g.C, g.gs, g.Kp,
+                                                               plan.w_bits == 4 ? 7 : 127);
         return cudaGetLastError();
     }
+}
+
+// 4-bit filter codes of the exported blob: byte j = code 2j in the low nibble, code 2j+1 in the
+// high nibble, two's complement.  One thread per 8 codes (two words in, one word out).
+namespace {
+__global__ void pack_nibbles_kernel(const uint2 *__restrict__ codes, uint32_t *__restrict__ packed, size_t words)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= words) return;
+    const uint2 c = codes[i];
+    uint32_t out = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        out |= ((c.x >> (8 * e)) & 0xfu) << (4 * e);
+        out |= ((c.y >> (8 * e)) & 0xfu) << (16 + 4 * e);
+    }
+    packed[i] = out;
+}
+
+__global__ void unpack_nibbles_kernel(const uint32_t *__restrict__ packed, uint2 *__restrict__ codes, size_t words)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= words) return;
+    const uint32_t w = packed[i];
+    uint2 c = make_uint2(0u, 0u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        // sign extension of a nibble: shift it to the top of an int, arithmetic shift back
+        const int lo = ((int)(w << (28 - 4 * e))) >> 28;
+        const int hi = ((int)(w << (12 - 4 * e))) >> 28;
+        c.x |= ((uint32_t)lo & 0xffu) << (8 * e);
+        c.y |= ((uint32_t)hi & 0xffu) << (8 * e);
+    }
+    codes[i] = c;
+}
+}  // namespace
+
+cudaError_t launch_pack_nibbles(const int8_t *codes, void *packed, size_t n_codes, cudaStream_t stream)
+{
+    const size_t words = n_codes / 8;
+    if (words == 0) return cudaSuccess;
+    pack_nibbles_kernel<<<(unsigned)((words + 255) / 256), 256, 0, stream>>>(
+        reinterpret_cast<const uint2 *>(codes), static_cast<uint32_t *>(packed), words);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack_nibbles(const void *packed, int8_t *codes, size_t n_codes, cudaStream_t stream)
+{
+    const size_t words = n_codes / 8;
+    if (words == 0) return cudaSuccess;
+    unpack_nibbles_kernel<<<(unsigned)((words + 255) / 256), 256, 0, stream>>>(
+        static_cast<const uint32_t *>(packed), reinterpret_cast<uint2 *>(codes), words);
+    return cudaGetLastError();
 }
 
 }  // namespace wfq
@@ -195,7 +251,7 @@ extern "C" wfq_status_t wfq_quantize_filters_static(const float *w_dev, int K, i
     {
         const long long total = (long long)P * K * (C / group_size);
         const unsigned blocks = (unsigned)((total + threads - 1) / threads);
-        filter_quantize_kernel<<<blocks, threads, 0, st>>>(w32, wq_dev, sw_dev, P, K, C, group_size, K);
+        filter_quantize_kernel<<<blocks, threads, 0, st>>>(w32, wq_dev, sw_dev, P, K, C, group_size, K, 127);
         if (cudaGetLastError() != cudaSuccess) return WFQ_ERR_CUDA;
     }
     return WFQ_OK;

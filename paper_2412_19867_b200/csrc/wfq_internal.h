@@ -103,6 +103,7 @@ struct wfq_plan {
     wfq::Workspace ws;
     bool has_workspace = false;
     bool prepared = false;
+    int w_bits = 8;            // bit width of the filter codes (8 or 4); the stored codes are int8 either way
     int device = -1;
     int sm_count = 0;
 
@@ -164,6 +165,9 @@ namespace wfq {
 // launch; none synchronises.
 cudaError_t launch_filter_prep(const wfq_plan &plan, const float *w_dev, float *scratch_w32,
                                cudaStream_t stream);
+// 4-bit filter codes <-> two codes per byte (the exported blob's storage); n_codes a multiple of 8
+cudaError_t launch_pack_nibbles(const int8_t *codes, void *packed, size_t n_codes, cudaStream_t stream);
+cudaError_t launch_unpack_nibbles(const void *packed, int8_t *codes, size_t n_codes, cudaStream_t stream);
 cudaError_t launch_input_transform(wfq_plan &plan, const void *x_dev, cudaStream_t stream);
 cudaError_t launch_input_transform_tc(const wfq_plan &plan, const void *x_dev, cudaStream_t stream);
 bool input_transform_tcn_applies(const wfq_plan &plan);

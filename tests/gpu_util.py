@@ -12,10 +12,12 @@ SCALE_RTOL = 1e-5              # fp32 group scales: fp32 transform vs fp64-then-
 FINAL_TOL = 2e-3               # max |y - y_ref| / max |y_ref|
 
 
-def make_conv(layer, tensors=None, device="cuda:0"):
+def make_conv(layer, tensors=None, device="cuda:0", w_bits=8):
     import torch
     x, w, sB, sG = wl.make_tensors(layer) if tensors is None else tensors
     conv = b.Conv(layer.N, layer.C, layer.K, layer.H, layer.W, layer.m, layer.gs, layer.dtype, device)
+    if w_bits != 8:
+        conv.set_weight_bits(w_bits)
     conv.prepare(torch.from_numpy(w).to(device), None if sB is None else list(sB),
                  None if sG is None else list(sG))
     return conv, (x, w, sB, sG)
@@ -55,14 +57,25 @@ def max_rel(got, want):
     return float(np.max(np.abs(np.asarray(got, dtype=np.float64) - want)) / max(np.max(np.abs(want)), 1e-300))
 
 
-def check_layer_all_levels(layer, tensors=None, final_tol=FINAL_TOL, k1_kernel=0):
+def oracle_wfq(x, w, layer, sB, sG, w_bits=8, **kw):
+    """The oracle's pipeline with the filters quantized to w_bits (activations: 8 bits)."""
+    filters = None
+    if w_bits != 8:
+        filters = orc.prepare_filters(w, layer.m, layer.gs, orc.matrices(layer.m, sB, sG, None), bits=w_bits)
+    return orc.wfq(x, w, layer.m, layer.gs, sB=sB, sG=sG, filters=filters, **kw)
+
+
+def check_layer_all_levels(layer, tensors=None, final_tol=FINAL_TOL, k1_kernel=0, w_bits=8):
     """Filters, stage 1, raw int32 group sums, stage 2, stage 3 and end to end.
-    k1_kernel: input-transform kernel (0 = the library's choice, 2 = tensor cores where they apply)."""
+    k1_kernel: input-transform kernel (0 = the library's choice, 2 = tensor cores where they apply);
+    w_bits: bit width of the filter codes."""
     import torch
-    conv, (x, w, sB, sG) = make_conv(layer, tensors)
+    conv, (x, w, sB, sG) = make_conv(layer, tensors, w_bits=w_bits)
     b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, k1_kernel)
     dev = conv.device
-    ref = orc.wfq(x, w, layer.m, layer.gs, sB=sB, sG=sG)
+    ref = oracle_wfq(x, w, layer, sB, sG, w_bits)
+    if w_bits != 8:
+        assert np.abs(ref.Wq).max() == 2 ** (w_bits - 1) - 1
     report = {}
 
     # offline filter path

@@ -111,9 +111,25 @@ def test_null_plan_is_rejected_everywhere(lib):
     assert lib.wfq_plan_set_epilogue(None, None, 0) == b.WFQ_ERR_INVALID_ARG
     assert lib.wfq_plan_set_output_dtype(None, 0) == b.WFQ_ERR_INVALID_ARG
     assert lib.wfq_plan_set_full_quant(None, 0, 0) == b.WFQ_ERR_INVALID_ARG
+    assert lib.wfq_plan_set_weight_bits(None, 8) == b.WFQ_ERR_INVALID_ARG
     assert lib.wfq_filters_bytes(None) == 0
     assert lib.wfq_filters_export(None, fake, 0, None) == b.WFQ_ERR_INVALID_ARG
     assert lib.wfq_filters_import(None, fake, 0, None) == b.WFQ_ERR_INVALID_ARG
+
+
+def test_weight_bits_and_blob_size(lib):
+    st, plan = _create(lib, 1, 64, 96, 8, 8, 4, 3, 32, 8)
+    assert st == b.WFQ_OK
+    full = lib.wfq_filters_bytes(plan)
+    codes, scales = 36 * 96 * 64, 36 * 2 * 128 * 4
+    assert full == 256 + codes + scales
+    for bits in (0, 2, 5, 16):
+        assert lib.wfq_plan_set_weight_bits(plan, bits) == b.WFQ_ERR_UNSUPPORTED
+    assert lib.wfq_plan_set_weight_bits(plan, 4) == b.WFQ_OK
+    assert lib.wfq_filters_bytes(plan) == 256 + codes // 2 + scales
+    assert lib.wfq_plan_set_weight_bits(plan, 8) == b.WFQ_OK
+    assert lib.wfq_filters_bytes(plan) == full
+    assert lib.wfq_plan_destroy(plan) == b.WFQ_OK
 
 
 def test_status_strings(lib):

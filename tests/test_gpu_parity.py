@@ -307,6 +307,77 @@ def test_filters_export_and_import():
     other.close(); same.close(); conv.close()
 
 
+W4_LAYERS = [
+    Layer(2, 64, 96, 18, 24, 2, 64, "f16", "silu_outlier", "kaiming_chan", 5, 9, 3),       # F(2,3)
+    Layer(3, 128, 128, 28, 28, 4, 32, "f16", "relu_heavy", "kaiming", 3, 0, 1),            # T=147
+    Layer(6, 128, 96, 14, 14, 6, 64, "f16", "relu_heavy", "kaiming", 2, 1, 1),             # ragged 14/6
+    Layer(1, 320, 64, 8, 8, 4, 160, "f16", "silu_outlier", "kaiming_chan", 4, 0, 8),       # swapped contraction
+    Layer(1, 256, 64, 20, 20, 4, 256, "f32", "gauss_outlier", "gauss_chan", 1, 0, 2),      # gs=256, fp32
+]
+
+
+@pytest.mark.parametrize("layer", W4_LAYERS, ids=lambda L: L.name)
+def test_four_bit_weights(layer):
+    """W4A8 (Section 5's naming: filter codes in [-7, 7], activations at 8 bits): every level of the
+    check against the oracle with its filters quantized to 4 bits, and the loss against W8A8 is
+    what the oracle shows."""
+    rep = _check(layer, w_bits=4)
+    x, w, sB, sG = wl.make_tensors(layer)
+    from oracle import oracle as orc
+    from tests import gpu_util as gu
+    direct = orc.direct(x, w)
+    want4 = orc.sqnr_db(direct, gu.oracle_wfq(x, w, layer, sB, sG, 4).y)
+    want8 = orc.sqnr_db(direct, gu.oracle_wfq(x, w, layer, sB, sG, 8).y)
+    assert abs(rep["sqnr_vs_direct_db"] - want4) <= 0.1, (rep, want4)
+    assert want4 < want8 - 10.0, (want4, want8)          # 4 bits fewer: about 24 dB in theory
+
+
+def test_four_bit_weights_blob_and_switching():
+    """The exported blob of a 4-bit plan stores two codes per byte (half the code section, the
+    documented nibble order), imports into a plan created for 8 bits, and switching the width
+    un-prepares the plan."""
+    import torch
+    from oracle import oracle as orc
+    from paper_2412_19867_b200 import binding as b
+    from tests import gpu_util as gu
+    L = Layer(2, 128, 72, 20, 24, 6, 64, "f16", "silu_outlier", "kaiming_chan", 9, 7, 1)
+    conv8, (x, w, sB, sG) = gu.make_conv(L)
+    conv4, _ = gu.make_conv(L, (x, w, sB, sG), w_bits=4)
+    codes = conv4.P * L.K * L.C
+    assert b.wfq_filters_bytes(conv8.plan) - b.wfq_filters_bytes(conv4.plan) == codes // 2
+    blob = bytes(b.wfq_filters_export(conv4.plan, conv4._stream()))
+    assert len(blob) == b.wfq_filters_bytes(conv4.plan)
+    ref = orc.prepare_filters(w, L.m, L.gs, orc.matrices(L.m, sB, sG, None), bits=4)
+    q = ref.Wq.reshape(-1).astype(np.int16)                               # [P][K][C], codes in [-7, 7]
+    packed = ((q[0::2] & 0xF) | ((q[1::2] & 0xF) << 4)).astype(np.uint8)
+    got = np.frombuffer(blob, dtype=np.uint8, count=codes // 2, offset=256)
+    assert np.mean(got != packed) <= gu.CODE_MISMATCH_RATE
+    xd = torch.from_numpy(x).to("cuda:0")
+    y4 = conv4.forward(xd).clone()
+    y8 = conv8.forward(xd).clone()
+    assert not torch.equal(y4, y8)
+    # a plan created for 8 bits takes the blob's width
+    c = b.Conv(L.N, L.C, L.K, L.H, L.W, L.m, L.gs, L.dtype)
+    b.wfq_filters_import(c.plan, blob, c._stream())
+    assert torch.equal(c.forward(xd), y4)
+    assert b.wfq_filters_bytes(c.plan) == len(blob)
+    c.check_status()
+    # a truncated 4-bit blob is refused
+    d = b.Conv(1, L.C, L.K, 8, 8, L.m, L.gs, L.dtype)
+    with pytest.raises(b.WfqError):
+        b.wfq_filters_import(d.plan, blob[:len(blob) - 16])
+    # switching the width: not prepared until the filters are quantized again; then 8-bit results
+    conv4.set_weight_bits(8)
+    with pytest.raises(b.WfqError):
+        conv4.forward(xd)
+    conv4.prepare(torch.from_numpy(w).to("cuda:0"), list(sB), list(sG))
+    assert torch.equal(conv4.forward(xd), y8)
+    with pytest.raises(b.WfqError):
+        conv4.set_weight_bits(5)
+    for o in (conv8, conv4, c, d):
+        o.close()
+
+
 def test_asynchronous_host_buffer_entry_point():
     """Two layers through wfq_conv_forward_host_async on two streams, repeatedly, against the
     synchronous entry point (one of them large enough for the chunked path)."""

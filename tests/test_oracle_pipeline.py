@@ -117,10 +117,55 @@ def test_quantizer_ties_round_half_to_even_and_idempotent():
     np.testing.assert_array_equal(q2[0].astype(np.float32), grid[0])
 
 
-def test_quantizer_other_bit_width():
+@pytest.mark.parametrize("bits", [4, 6])
+def test_quantizer_other_bit_widths_brute_force(bits):
+    """The same quantizer with 2^(bits-1) - 1 in place of 127 (4 bits: the weight side of the
+    W4A8 setting, Section 5): scale, every code by brute force, error at most half a step."""
+    qmax = 2 ** (bits - 1) - 1
     v = np.linspace(-1, 1, 32, dtype=np.float32)[None, :]
-    q, s = orc.quantize_groups(v, 32, bits=4)
-    assert q.max() == 7 and q.min() == -7 and s[0, 0] == np.float32(1.0) / np.float32(7.0)
+    q, s = orc.quantize_groups(v, 32, bits=bits)
+    assert q.max() == qmax and q.min() == -qmax and s[0, 0] == np.float32(1.0) / np.float32(qmax)
+    rng = np.random.default_rng(50 + bits)
+    v = rng.standard_normal((5, 64)).astype(np.float32) * np.float32(0.37)
+    v[1, 32:] = 0.0
+    v[2, 7] = 55.0
+    q, s = orc.quantize_groups(v, 32, bits=bits)
+    for r in range(5):
+        for g in range(2):
+            grp = v[r, 32 * g:32 * g + 32]
+            amax = np.max(np.abs(grp))
+            if amax == 0:
+                assert s[r, g] == 0 and not q[r, 32 * g:32 * g + 32].any()
+                continue
+            scale = np.float32(amax) / np.float32(qmax)
+            inv = np.float32(qmax) / np.float32(amax)
+            assert s[r, g] == scale
+            want = [int(np.clip(np.rint(np.float32(e) * inv), -qmax, qmax)) for e in grp]
+            assert list(q[r, 32 * g:32 * g + 32]) == want
+            assert np.max(np.abs(want)) == qmax
+            assert np.all(np.abs(grp - np.float64(scale) * np.array(want)) <= 0.5 * scale * (1 + 1e-5))
+    # ties at inv = 1: half to even, as at 8 bits
+    t = np.zeros((1, 32), dtype=np.float32)
+    t[0, :6] = [qmax, 0.5, 1.5, 2.5, -0.5, -1.5]
+    q, s = orc.quantize_groups(t, 32, bits=bits)
+    assert s[0, 0] == 1.0 and list(q[0, :6]) == [qmax, 0, 2, 2, 0, -2]
+
+
+def test_four_bit_filters_cost_about_four_bits_of_sqnr():
+    """Filters at 4 bits with activations at 8 (through `filters=`): the error of the result is
+    dominated by the filter codes' step, 127/7 = 18 times coarser, so the SQNR against the direct
+    convolution falls by about 20 log10(18) = 25 dB (within a few dB on random data)."""
+    from paper_2412_19867_b200 import workloads as wl
+    L = wl.Layer(1, 64, 32, 12, 12, 4, 32, "f32", "gauss", "kaiming", 8, 11, 0)
+    x, w, sB, sG = wl.make_tensors(L)
+    direct = orc.direct(x, w)
+    f4 = orc.prepare_filters(w, L.m, L.gs, orc.matrices(L.m, sB, sG, None), bits=4)
+    assert np.abs(f4.Wq).max() == 7
+    r8 = orc.wfq(x, w, L.m, L.gs, sB, sG)
+    r4 = orc.wfq(x, w, L.m, L.gs, sB, sG, filters=f4)
+    assert np.array_equal(r4.Xq, r8.Xq)                       # the activation side is untouched
+    drop = orc.sqnr_db(direct, r8.y) - orc.sqnr_db(direct, r4.y)
+    assert 18.0 <= drop <= 30.0, drop
 
 
 def test_contract_matches_integer_einsum_and_bound():
