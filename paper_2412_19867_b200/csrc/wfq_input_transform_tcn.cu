@@ -38,12 +38,16 @@
 namespace wfq {
 namespace {
 
-constexpr int TN_THREADS = 256;
+// quantizer teams of four warps; team k takes the CTA's items k, k + TEAMS, ...  (a second team, one per
+// accumulator, and a fourth strip were measured: no difference on any configured layer)
+constexpr int TN_TEAMS = 1;
+constexpr int TN_FIRST_QUANT = 4;
+constexpr int TN_THREADS = 32 * (TN_FIRST_QUANT + 4 * TN_TEAMS);
 constexpr int TN_CB = 64;             // channels per work item = columns of the accumulator
 constexpr int TN_NSTRIP = 3;          // strip ring
 constexpr int TN_NACC = 2;            // accumulators
 constexpr int TN_TMEM_COLS = TN_NACC * TN_CB;
-constexpr int TN_FIRST_QUANT = 4;
+static_assert(TN_TEAMS == 1 || TN_TEAMS == TN_NACC, "a team owns an accumulator, or one team takes them in turn");
 
 template <int M>
 struct TnCfg {
@@ -205,9 +209,11 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
         const bool row_ok = tl < C::TB && p < C::P;
         const float sp = row_ok ? tab.in_scale[p] : 0.f, sl = row_ok ? tab.in_scale_lo[p] : 0.f;
         const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        int slot = 0;
+        // one team: both accumulators in turn; two teams: team k owns accumulator k
+        const int team = (warp - TN_FIRST_QUANT) >> 2;
+        int slot = TN_TEAMS == 1 ? 0 : team;
         uint32_t aphase = 0;
-        for (int item = blockIdx.x; item < a.items; item += stride) {
+        for (int item = blockIdx.x + team * stride; item < a.items; item += TN_TEAMS * stride) {
             if (!wait_bounded(ptx::smem_u32(&sh.acc_full[slot]), aphase, ctx, kWaitAccFull)) break;
             ptx::tc_fence_after();
             const int cblk = item % a.NCB, rest = item / a.NCB;
@@ -257,7 +263,11 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.acc_empty[slot]));
                 if (valid) codes32(v, sp, sl, inv, dst);
             }
-            if (++slot == TN_NACC) { slot = 0; aphase ^= 1u; }
+            if (TN_TEAMS == 1) {
+                if (++slot == TN_NACC) { slot = 0; aphase ^= 1u; }
+            } else {
+                aphase ^= 1u;
+            }
         }
     }
 
