@@ -283,7 +283,7 @@ class Workload:
     """The layers of one configuration: plans, device tensors, and the step as a CUDA graph."""
 
     def __init__(self, cfg, only_layer, dev, stream, flush, use_graph=True, k1_kernel=0, full_quant=None,
-                 nhwc=False):
+                 nhwc=False, streams=1):
         import torch
         from paper_2412_19867_b200 import binding as b
         from paper_2412_19867_b200 import workloads as wl
@@ -308,6 +308,9 @@ class Workload:
             self.ys.append(torch.empty((L.N, L.K, L.H, L.W), dtype=torch.float32, device=dev))
         self.step_ops = float(sum(L.direct_ops for L in self.layers))
         self.sptr = stream.cuda_stream
+        # streams > 1: the layers (independent problems, each with its own plan and workspace) are
+        # dealt round-robin onto that many streams forked from and joined to the launching stream
+        self.extra = [torch.cuda.Stream(dev) for _ in range(streams - 1)] if streams > 1 else []
         # One step = the forward calls of all layers.  They are captured once into a CUDA
         # graph and replayed (same kernels, same order, one submission per step); stream
         # launches are the fallback and what --no-graph selects.
@@ -320,16 +323,26 @@ class Workload:
                 side.wait_stream(stream)
                 cand = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(cand, stream=side):
-                    self.enqueue(side.cuda_stream)
+                    self.enqueue(side.cuda_stream, side)
                 torch.cuda.synchronize(dev)
                 self.graph, self.launch_mode = cand, "CUDA graph replay"
             except Exception as exc:   # capture is an optimisation of the submission only
                 print(f"bench: graph capture failed ({exc!r}); using stream launches", file=sys.stderr)
                 torch.cuda.synchronize(dev)
 
-    def enqueue(self, stream_ptr):
-        for conv, x, y in zip(self.convs, self.xs, self.ys):
-            self.b.wfq_conv_forward(conv.plan, x.data_ptr(), y.data_ptr(), stream_ptr)
+    def enqueue(self, stream_ptr, main=None):
+        if not self.extra:
+            for conv, x, y in zip(self.convs, self.xs, self.ys):
+                self.b.wfq_conv_forward(conv.plan, x.data_ptr(), y.data_ptr(), stream_ptr)
+            return
+        main = self.stream if main is None else main
+        lanes = [main] + self.extra
+        for s in self.extra:
+            s.wait_stream(main)
+        for i, (conv, x, y) in enumerate(zip(self.convs, self.xs, self.ys)):
+            self.b.wfq_conv_forward(conv.plan, x.data_ptr(), y.data_ptr(), lanes[i % len(lanes)].cuda_stream)
+        for s in self.extra:
+            main.wait_stream(s)
 
     def step(self):
         if self.graph is not None:
@@ -808,19 +821,45 @@ def run_wfq(args):
             torch.cuda.synchronize(dev)
             ms = [statistics.median(w4.timed_replays(reps)) for _ in range(10)]
             s4, _, _ = w4.summary(statistics.mean(ms), w4.kernel_split(10), peak)
-            # the tensor-core transform rounds V in another order than the NCHW kernel: a code in about
-            # 1e-6 may differ by one step, so the outputs are compared in norm, not bit for bit
+            # the tensor cores accumulate V in another order than the NCHW kernel's add/fma chains: group
+            # scales differ in the last bit, and a code in about a million by one step (which moves its tile
+            # by a quantization step: visible in the norm on the F(6,3) layers), so the outputs are compared
+            # in norm with each other and, like the headline's, with the oracle on sampled tiles
             dev_rel = max(float(torch.linalg.vector_norm(a.float() - b_.float()) /
                                 torch.linalg.vector_norm(b_.float())) for a, b_ in zip(w4.ys, ys_headline))
             nhwc = {"workload": s4["workload"], "value": s4["value"], "unit": UNIT, "us_per_step": s4["us_per_step"],
                     "input_transform_us_per_step": s4["kernels"][KERNELS[0]]["us_per_step"],
                     "kernel": "input_transform_tcn_kernel (TMA box as the MN-major operand of tcgen05.mma kind::f16)",
-                    "rel_l2_vs_nchw_result": dev_rel, "agrees_with_nchw_result": bool(dev_rel <= 1e-4)}
+                    "parity": w4.parity(), "worst_rel_l2_vs_nchw_result": dev_rel}
             w4.close()
             del w4
             torch.cuda.empty_cache()
         except Exception as exc:
             nhwc = {"error": repr(exc)}
+
+    # ---- the headline workload with its layers on three streams, reported beside ----
+    concurrent = None
+    if rank == 0 and world == 1 and not args.no_extras and args.only_layer is None:
+        try:
+            w5 = Workload(args.config, None, dev, stream, flush, use_graph=not args.no_graph, streams=3)
+            for _ in range(3):
+                flush.zero_()
+                w5.step()
+            torch.cuda.synchronize(dev)
+            w5.check()
+            ms = statistics.mean(statistics.median(w5.timed_replays(reps)) for _ in range(10))
+            same = all(torch.equal(a, b_) for a, b_ in zip(w5.ys, ys_headline))
+            concurrent = {"streams": 3, "value": w5.step_ops / (ms * 1e-3) / 1e12, "unit": UNIT,
+                          "us_per_step": ms * 1e3, "equals_serial_result": bool(same),
+                          "note": "the layers of a step are independent problems: dealt round-robin onto three "
+                                  "streams inside the replayed graph, so that one layer's latency-bound input and "
+                                  "output transforms overlap another layer's contraction; the headline keeps them "
+                                  "in one stream, which is what the per-kernel split needs"}
+            w5.close()
+            del w5
+            torch.cuda.empty_cache()
+        except Exception as exc:
+            concurrent = {"error": repr(exc)}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -840,7 +879,7 @@ def run_wfq(args):
                            "parallelism": "replicas" if world > 1 else "single GPU"},
                 "timing": timing, "us_per_layer": head["us_per_layer"], "wall_s_timed_region": wall,
                 "warm": warm, "sustained": sustained, "roofline": roofline, "contraction": contraction,
-                "parity": parity, "per_config": per_config, "full_quant": full_quant, "nhwc_input": nhwc, "cpu_baseline": cpu, "e2e": e2e,
+                "parity": parity, "per_config": per_config, "full_quant": full_quant, "nhwc_input": nhwc, "layers_on_three_streams": concurrent, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": 3 * len(layers) * args.steps * reps, "clocks": clocks}
         print(json.dumps(line), flush=True)
     if world > 1:

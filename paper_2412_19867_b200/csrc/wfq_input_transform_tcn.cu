@@ -113,23 +113,31 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmx);
     }
-    if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TN_TMEM_COLS);
-        ptx::tmem_relinquish();
+    __syncthreads();                    // the barriers exist
+    uint32_t tmem_base = 0;
+    if (warp == 0) {
+        // the producer needs neither the A operand nor TMEM: its first boxes are in flight while the
+        // other warps set those up
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    } else {
+        if (warp == 1) {
+            ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TN_TMEM_COLS);
+            ptx::tmem_relinquish();
+        }
+        // the A operand: zero rows, the constant matrix (a plain copy; it does not depend on the previous
+        // kernel), zero rows
+        for (int i = threadIdx.x - 32; i < C::A_BYTES / 16; i += TN_THREADS - 32) {
+            const int j = i - C::Z0 * 8;                           // 16-byte pieces: 8 per row
+            reinterpret_cast<uint4 *>(amat_s)[i] =
+                (j >= 0 && j < C::AMAT_BYTES / 16) ? __ldg(a.amat + j) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        ptx::fence_proxy_async_smem();      // the tensor cores read it through the async proxy
+        ptx::tc_fence_before();
+        asm volatile("bar.sync 1, %0;" ::"n"(TN_THREADS - 32) : "memory");      // warps 1 ..: operand and TMEM ready
+        ptx::tc_fence_after();
+        tmem_base = sh.tmem_base;
+        asm volatile("griddepcontrol.wait;" ::: "memory");
     }
-    // the A operand: zero rows, the constant matrix (a plain copy; it does not depend on the previous
-    // kernel), zero rows
-    for (int i = threadIdx.x; i < C::A_BYTES / 16; i += TN_THREADS) {
-        const int j = i - C::Z0 * 8;                           // 16-byte pieces: 8 per row
-        reinterpret_cast<uint4 *>(amat_s)[i] =
-            (j >= 0 && j < C::AMAT_BYTES / 16) ? __ldg(a.amat + j) : make_uint4(0u, 0u, 0u, 0u);
-    }
-    ptx::fence_proxy_async_smem();      // the tensor cores read it through the async proxy
-    ptx::tc_fence_before();
-    __syncthreads();
-    ptx::tc_fence_after();
-    const uint32_t tmem_base = sh.tmem_base;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int stride = (int)gridDim.x;
     if (warp == 0) {
