@@ -222,6 +222,11 @@ def test_contraction_shapes_agree(layer):
     Layer(2, 64, 32, 10, 14, 2, 64, "f16", "silu_outlier", "kaiming_chan", 9, 8, 7),      # F(2,3)
     Layer(2, 128, 32, 21, 26, 4, 32, "f16", "silu_outlier", "kaiming_chan", 9, 8, 8),     # tensor cores, F(4,3), groups of 32
     Layer(1, 320, 32, 64, 64, 4, 64, "f16", "silu_outlier", "kaiming_chan", 9, 8, 9),     # tensor cores, several items per CTA
+    # tensor cores: images narrower than the 8-column box, tile rows shorter than a work item
+    # (whole tiles of the item outside the image), an odd number of tile columns, groups of 32 with F(6,3)
+    Layer(9, 128, 32, 7, 7, 6, 64, "f16", "relu_heavy", "kaiming", 9, 8, 10),
+    Layer(2, 64, 32, 5, 5, 4, 32, "f16", "silu_outlier", "kaiming_chan", 9, 8, 11),
+    Layer(3, 128, 40, 30, 18, 6, 32, "f16", "silu_outlier", "kaiming_chan", 9, 8, 12),
 ], ids=lambda L: L.name)
 def test_nhwc_input_matches_nchw(layer):
     """x given as [N][H][W][C].  With the plain NHWC kernel (TMA-staged strips, debug option 1) the
