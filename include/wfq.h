@@ -61,7 +61,7 @@ typedef enum {
     WFQ_ERR_SCRATCH_TOO_SMALL = 7 /* problem larger than the library's built-in scratch */
 } wfq_status_t;
 
-typedef enum { WFQ_F32 = 0, WFQ_F16 = 1 } wfq_dtype_t;
+typedef enum { WFQ_F32 = 0, WFQ_F16 = 1, WFQ_BF16 = 2 /* output only */ } wfq_dtype_t;
 
 /* Memory layout of the input x: [N][C][H][W] (default) or [N][H][W][C]. */
 typedef enum { WFQ_NCHW = 0, WFQ_NHWC = 1 } wfq_layout_t;
@@ -141,10 +141,11 @@ wfq_status_t wfq_plan_set_epilogue(wfq_plan_t *plan, const float *bias_dev, wfq_
 wfq_status_t wfq_plan_set_input_layout(wfq_plan_t *plan, wfq_layout_t layout);
 
 /*
- * Element type of the output y: WFQ_F32 (default) or WFQ_F16.  With WFQ_F16 the output transform
- * rounds each result once to fp16 (after bias and activation) and `y_nkhw_dev` / `y_host` of the
- * forward calls point at fp16 storage of the same [N][K][H][W] shape (the parameters keep their
- * `float *` type; alignment requirements are unchanged).  Host only.
+ * Element type of the output y: WFQ_F32 (default), WFQ_F16 or WFQ_BF16.  With a 16-bit type the
+ * output transform rounds each result once (to nearest even, after bias and activation) and
+ * `y_nkhw_dev` / `y_host` of the forward calls point at 2-byte storage of the same [N][K][H][W]
+ * shape (the parameters keep their `float *` type; alignment requirements are unchanged).
+ * Host only.
  */
 wfq_status_t wfq_plan_set_output_dtype(wfq_plan_t *plan, wfq_dtype_t dtype);
 

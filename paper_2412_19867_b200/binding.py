@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libwfq.so")
 WFQ_OK, WFQ_ERR_INVALID_ARG, WFQ_ERR_UNSUPPORTED, WFQ_ERR_ALLOC = 0, 1, 2, 3
 WFQ_ERR_NOT_PREPARED, WFQ_ERR_CUDA, WFQ_ERR_TIMEOUT, WFQ_ERR_SCRATCH_TOO_SMALL = 4, 5, 6, 7
 WFQ_STATIC_SCRATCH_FLOATS = 4 * 1024 * 1024
-WFQ_F32, WFQ_F16 = 0, 1
+WFQ_F32, WFQ_F16, WFQ_BF16 = 0, 1, 2
 WFQ_ACT_NONE, WFQ_ACT_RELU, WFQ_ACT_SILU = 0, 1, 2
 WFQ_Y_FP32, WFQ_Y_TILE, WFQ_Y_ROW = 0, 1, 2
 WFQ_NCHW, WFQ_NHWC = 0, 1
@@ -294,9 +294,9 @@ class Conv:
         wfq_plan_set_weight_bits(self.plan, bits)
 
     def set_output_dtype(self, dtype):
-        """"f32" (default) or "f16": element type of the tensors forward() returns or fills."""
+        """"f32" (default), "f16" or "bf16": element type of the tensors forward() returns or fills."""
         self.out_dtype = dtype
-        wfq_plan_set_output_dtype(self.plan, WFQ_F16 if dtype == "f16" else WFQ_F32)
+        wfq_plan_set_output_dtype(self.plan, {"f32": WFQ_F32, "f16": WFQ_F16, "bf16": WFQ_BF16}[dtype])
 
     def set_epilogue(self, bias=None, act=WFQ_ACT_NONE):
         """bias: fp32 CUDA tensor [K] or None; kept alive by this object."""
@@ -312,7 +312,7 @@ class Conv:
         xs = (N, H, W, C) if getattr(self, "in_layout", "nchw") == "nhwc" else (N, C, H, W)
         assert x.is_cuda and x.is_contiguous() and tuple(x.shape) == xs
         assert x.dtype == (torch.float16 if self.in_dtype == "f16" else torch.float32)
-        ydt = torch.float16 if getattr(self, "out_dtype", "f32") == "f16" else torch.float32
+        ydt = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[getattr(self, "out_dtype", "f32")]
         if y is None:
             y = torch.empty((N, K, H, W), dtype=ydt, device=self.device)
         assert y.dtype == ydt and y.is_contiguous() and tuple(y.shape) == (N, K, H, W)

@@ -225,8 +225,8 @@ size_t wfq_plan_workspace_bytes(const wfq_plan_t *plan) { return plan ? plan->ws
 
 wfq_status_t wfq_plan_set_output_dtype(wfq_plan_t *plan, wfq_dtype_t dtype)
 {
-    if (!plan || (dtype != WFQ_F32 && dtype != WFQ_F16)) return WFQ_ERR_INVALID_ARG;
-    plan->out_half = dtype == WFQ_F16;
+    if (!plan || (dtype != WFQ_F32 && dtype != WFQ_F16 && dtype != WFQ_BF16)) return WFQ_ERR_INVALID_ARG;
+    plan->out_half = dtype == WFQ_F16 ? 1 : dtype == WFQ_BF16 ? 2 : 0;
     plan->host_chunks = 0;         // chunk sizes of the host-buffer path depend on the output bytes
     for (int i = 0; i < 2; ++i)
         if (plan->sub[i]) plan->sub[i]->out_half = plan->out_half;

@@ -18,6 +18,7 @@
 // matrix products as plain multiply-adds with the codes of the matrices as kernel parameters.
 #include <cmath>
 
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "wfq_internal.h"
@@ -253,7 +254,8 @@ output_transform_int_kernel(const float *__restrict__ Y, float *__restrict__ y, 
                 float r = (float)out[u][c] + bk;
                 if (act == 1) r = fmaxf(r, 0.f);
                 else if (act == 2) r = r * __frcp_rn(1.f + __expf(-r));
-                if (out_half) reinterpret_cast<__half *>(y)[(dst - y) + (size_t)u * g.W + c] = __float2half_rn(r);
+                if (out_half == 2) reinterpret_cast<__nv_bfloat16 *>(y)[(dst - y) + (size_t)u * g.W + c] = __float2bfloat16_rn(r);
+                else if (out_half) reinterpret_cast<__half *>(y)[(dst - y) + (size_t)u * g.W + c] = __float2half_rn(r);
                 else dst[(size_t)u * g.W + c] = r;
             }
 }
@@ -362,13 +364,13 @@ cudaError_t launch_output_transform_int(const wfq_plan &plan, float *y_dev, cuda
     const dim3 grid((unsigned)((g.T + 127) / 128), (unsigned)g.K), block(128);
     const float *Y = plan.ws.Y;
     if (plan.fq_output == 1) {
-        if (g.m == 2) output_transform_int_kernel<2, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
-        else if (g.m == 4) output_transform_int_kernel<4, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
-        else output_transform_int_kernel<6, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
+        if (g.m == 2) output_transform_int_kernel<2, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half);
+        else if (g.m == 4) output_transform_int_kernel<4, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half);
+        else output_transform_int_kernel<6, 1><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half);
     } else {
-        if (g.m == 2) output_transform_int_kernel<2, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
-        else if (g.m == 4) output_transform_int_kernel<4, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
-        else output_transform_int_kernel<6, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half ? 1 : 0);
+        if (g.m == 2) output_transform_int_kernel<2, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half);
+        else if (g.m == 4) output_transform_int_kernel<4, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half);
+        else output_transform_int_kernel<6, 2><<<grid, block, 0, stream>>>(Y, y_dev, g, plan.fq, plan.bias, plan.act, plan.out_half);
     }
     return cudaGetLastError();
 }

@@ -113,7 +113,7 @@ struct wfq_plan {
     int *status = nullptr;     // int32[4]
     const float *bias = nullptr;   // caller-owned fp32[K] added in the output transform, or null
     int act = 0;               // activation after the bias: 0 none, 1 ReLU, 2 SiLU
-    bool out_half = false;     // y is written as fp16 instead of fp32
+    int out_half = 0;          // y is written as fp32 (0), fp16 (1) or bf16 (2)
     void *x_stage = nullptr;   // staging for wfq_conv_forward_host
     float *y_stage = nullptr;
 

@@ -3,6 +3,7 @@
 // Y[P][K][Tp] are 128-byte coalesced; the m-float row segments of neighbouring tiles are
 // contiguous in y[N][K][H][W] and are written in whole sectors.  P*4 bytes read
 // and m*m*4 bytes written per thread against ~150 flops.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "wfq_internal.h"
@@ -10,6 +11,16 @@
 
 namespace wfq {
 namespace {
+
+// One rounding to the 16-bit output type: kind 1 = fp16, 2 = bf16 (round to nearest even).
+__device__ __forceinline__ uint16_t to_bits16(float v, int kind)
+{
+    return kind == 2 ? __bfloat16_as_ushort(__float2bfloat16_rn(v)) : __half_as_ushort(__float2half_rn(v));
+}
+__device__ __forceinline__ uint32_t to_bits16x2(float lo, float hi, int kind)
+{
+    return (uint32_t)to_bits16(lo, kind) | ((uint32_t)to_bits16(hi, kind) << 16);
+}
 
 // F(2,3), points 0, 1, -1, inf: V_A = [1,1,1,0; 0,1,-1,1] (the sign of the textbook's last column is
 // in the standard S_A).
@@ -82,8 +93,9 @@ __global__ void __launch_bounds__(128, M == 6 ? (EPI ? 6 : 7) : 8)
 output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geometry g,
                         ScaleTables tab, const float *__restrict__ bias, int act, int out_half)
 {
-    // fp16 output (epilogue variants only): y points at __half storage of the same shape
-    [[maybe_unused]] __half *yh = reinterpret_cast<__half *>(y);
+    // 16-bit output (epilogue variants only; out_half 1 = fp16, 2 = bf16): y points at 2-byte storage
+    // of the same shape
+    [[maybe_unused]] uint16_t *yh = reinterpret_cast<uint16_t *>(y);
     constexpr int NN = M + 2;
     constexpr int TT = 128;                       // tiles per CTA
     __shared__ __align__(16) float out_s[STORE != 2 ? M * TT * M : 1];   // [u][tile][v]
@@ -162,7 +174,7 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
                     const int lim = tile_lim[tj];
                     if (u < (lim >> 4) && v1 < (lim & 15)) {
                         const size_t off = (size_t)tile_base[tj] + (size_t)u * g.W + v1;
-                        if (EPI && out_half) yh[off] = __float2half_rn(row[f]);
+                        if (EPI && out_half) yh[off] = to_bits16(row[f], out_half);
                         else y[off] = row[f];
                     }
                 }
@@ -181,14 +193,14 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
                 const int lim = tile_lim[tj];
                 if (u < (lim >> 4) && v2 < (lim & 15)) {    // W even: both columns or none
                     const size_t off = (size_t)tile_base[tj] + (size_t)u * g.W + v2;
-                    if (EPI && out_half) *reinterpret_cast<__half2 *>(yh + off) = __float22half2_rn(row[q]);
+                    if (EPI && out_half) *reinterpret_cast<uint32_t *>(yh + off) = to_bits16x2(row[q].x, row[q].y, out_half);
                     else *reinterpret_cast<float2 *>(y + off) = row[q];
                 }
             }
         }
     } else {
         float *row = y + base;
-        __half *rowh = yh + base;
+        uint16_t *rowh = yh + base;
         const bool full_w = (w0 + M <= g.W);
         const float bk = (EPI && bias) ? __ldg(bias + k) : 0.f;
 #pragma unroll
@@ -199,13 +211,12 @@ output_transform_kernel(const float *__restrict__ Y, float *__restrict__ y, Geom
             if (h0 + u < g.H) {
                 if (EPI && out_half) {
                     if (full_w) {
-                        const __half2 lo = __floats2half2_rn(o[0], o[1]), hi = __floats2half2_rn(o[2], o[3]);
-                        *reinterpret_cast<uint2 *>(rowh) = make_uint2(*reinterpret_cast<const uint32_t *>(&lo),
-                                                                      *reinterpret_cast<const uint32_t *>(&hi));
+                        *reinterpret_cast<uint2 *>(rowh) = make_uint2(to_bits16x2(o[0], o[1], out_half),
+                                                                      to_bits16x2(o[2], o[3], out_half));
                     } else {
 #pragma unroll
                         for (int v2 = 0; v2 < M; ++v2)
-                            if (w0 + v2 < g.W) rowh[v2] = __float2half_rn(o[v2]);
+                            if (w0 + v2 < g.W) rowh[v2] = to_bits16(o[v2], out_half);
                     }
                 } else if (full_w) {
                     *reinterpret_cast<float4 *>(row) = make_float4(o[0], o[1], o[2], o[3]);
@@ -236,7 +247,7 @@ template <int M, int STORE>
 cudaError_t launch_variant(const cudaLaunchConfig_t &cfg, const wfq_plan &plan, float *y_dev)
 {
     const float *Y = plan.ws.Y;
-    const int out_half = plan.out_half ? 1 : 0;
+    const int out_half = plan.out_half;
     if (plan.bias || plan.act || out_half)
         return cudaLaunchKernelEx(&cfg, output_transform_kernel<M, STORE, true>, Y, y_dev, plan.geo, plan.tables,
                                   plan.bias, plan.act, out_half);

@@ -87,6 +87,10 @@ def test_workspace_size_and_order_of_calls(lib):
     assert lib.wfq_plan_set_workspace(plan, ctypes.c_void_p(1024), want - 1) == b.WFQ_ERR_INVALID_ARG
     assert lib.wfq_plan_set_workspace(plan, ctypes.c_void_p(1024 + 16), want) == b.WFQ_ERR_INVALID_ARG
     assert lib.wfq_plan_set_input_dtype(plan, 7) == b.WFQ_ERR_INVALID_ARG
+    assert lib.wfq_plan_set_input_dtype(plan, b.WFQ_BF16) == b.WFQ_ERR_INVALID_ARG     # bf16: output only
+    assert lib.wfq_plan_set_output_dtype(plan, 3) == b.WFQ_ERR_INVALID_ARG
+    for dt in (b.WFQ_BF16, b.WFQ_F16, b.WFQ_F32):
+        assert lib.wfq_plan_set_output_dtype(plan, dt) == b.WFQ_OK
     assert lib.wfq_plan_set_input_dtype(plan, b.WFQ_F16) == b.WFQ_OK
     assert lib.wfq_prepare_filters(plan, None, None, None, None, None) == b.WFQ_ERR_INVALID_ARG
     # a zero or non-finite scale is rejected before any device work

@@ -154,8 +154,8 @@ def test_bias_and_activation_epilogue(m, H, W):
 @pytest.mark.parametrize("m,H,W", [(4, 16, 16), (4, 9, 14), (4, 7, 7), (6, 12, 12), (6, 13, 11), (2, 8, 10), (2, 7, 9)],
                          ids=["f43_w16", "f43_w14", "f43_w7", "f63_w12", "f63_w11", "f23_w10", "f23_w9"])
 def test_fp16_output(m, H, W):
-    """y written as fp16 by every store variant equals the fp32 result rounded once, with and
-    without an epilogue, through the device and the host-buffer entry points, and in the
+    """y written as fp16 or bf16 by every store variant equals the fp32 result rounded once, with
+    and without an epilogue, through the device and the host-buffer entry points, and in the
     fully quantized mode."""
     import torch
     from paper_2412_19867_b200 import binding as b
@@ -170,15 +170,16 @@ def test_fp16_output(m, H, W):
             b.wfq_plan_set_full_quant(conv.plan, *fq_mode)
             conv.set_output_dtype("f32")
             y32 = conv.forward(xd)
-            conv.set_output_dtype("f16")
-            y16 = conv.forward(xd)
-            conv.check_status()
-            assert y16.dtype == torch.float16
-            assert torch.equal(y16, y32.to(torch.float16)), (epi, fq_mode)
-            xh = torch.from_numpy(x).pin_memory()
-            yh = torch.empty(y16.shape, dtype=torch.float16).pin_memory()
-            conv.forward_host(xh, yh)
-            assert torch.equal(yh, y16.cpu())
+            for name, dt in (("f16", torch.float16), ("bf16", torch.bfloat16)):
+                conv.set_output_dtype(name)
+                y16 = conv.forward(xd)
+                conv.check_status()
+                assert y16.dtype == dt
+                assert torch.equal(y16, y32.to(dt)), (epi, fq_mode, name)
+                xh = torch.from_numpy(x).pin_memory()
+                yh = torch.empty(y16.shape, dtype=dt).pin_memory()
+                conv.forward_host(xh, yh)
+                assert torch.equal(yh, y16.cpu())
     conv.close()
 
 
