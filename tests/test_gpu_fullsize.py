@@ -26,13 +26,27 @@ def test_full_size_sampled_tiles_tensor_core_input_transform(layer):
     test_full_size_sampled_tiles(layer, k1_kernel=2)
 
 
+# NHWC input at full size (the tensor-core kernel that takes the TMA boxes as operands; groups of 128
+# go to the plain NHWC kernel): both tile sizes, groups of 32 / 64 / 128, one and many items per CTA
+NHWC_FULL = ([wl.config_layers(5)[i] for i in (0, 4, 5, 9)] + [wl.config_layers(2)[i] for i in (0, 3)] +
+             [wl.config_layers(3)[i] for i in (0, 8, 9)])
+
+
+@pytest.mark.parametrize("layer", NHWC_FULL, ids=lambda L: L.name)
+def test_full_size_sampled_tiles_nhwc_input(layer):
+    test_full_size_sampled_tiles(layer, nhwc=True)
+
+
 @pytest.mark.parametrize("layer", FULL, ids=lambda L: L.name)
-def test_full_size_sampled_tiles(layer, k1_kernel=0):
+def test_full_size_sampled_tiles(layer, k1_kernel=0, nhwc=False):
     import torch
     from tests.gpu_util import make_conv, codes_close, scales_close, max_rel, FINAL_TOL
     conv, (x, w, sB, sG) = make_conv(layer)
     b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, k1_kernel)
     xd = torch.from_numpy(x).cuda()
+    if nhwc:
+        conv.set_input_layout("nhwc")
+        xd = xd.permute(0, 2, 3, 1).contiguous()
     y = conv.forward(xd)
     torch.cuda.synchronize()
     conv.check_status()
