@@ -18,9 +18,15 @@
 // thread then owns one (tile, position) and reads its 64 channels with tcgen05.ld: abs-max over
 // registers, scale, 64 contiguous codes; no im2col, no fp32 round trip through shared memory.
 //
-// Persistent CTAs, two per SM, 8 warps:
+// A work item is TB tiles x one channel group of 64, 128 or 256 channels (or two groups of 32): a group of
+// 128 / 256 channels is 2 / 4 boxes per tile whose MMAs fill neighbouring 64-column blocks of the same
+// accumulator, and its quantizer threads take the abs-max over all those columns before the codes.
+//
+// Persistent CTAs, two per SM (one for groups of 256: two accumulators of 256 columns are all of tensor
+// memory), 8 warps:
 //   warp 0     TMA producer: per work item TB boxes (one per tile; tiles past the end of the tile
-//              row are loaded all the same and come back as zeros) into a ring of three strips
+//              row are loaded all the same and come back as zeros) into a ring of three strips (two for
+//              groups of 128 and 256)
 //   warp 1     owns TMEM; one lane issues TB * n / 2 MMAs per item (M = 128, N = 64, K = 16) into one
 //              of two accumulators of 64 columns, commits the accumulator and the strip
 //   warps 4-7  quantizers: warp % 4 selects the 32 TMEM lanes; per-position factor, abs-max, scale,
@@ -43,14 +49,21 @@ namespace {
 constexpr int TN_TEAMS = 1;
 constexpr int TN_FIRST_QUANT = 4;
 constexpr int TN_THREADS = 32 * (TN_FIRST_QUANT + 4 * TN_TEAMS);
-constexpr int TN_CB = 64;             // channels per work item = columns of the accumulator
-constexpr int TN_NSTRIP = 3;          // strip ring
+constexpr int TN_CB = 64;             // channels per box = N of one MMA
+constexpr int TN_MAX_NSTRIP = 3;      // strip ring (at most)
 constexpr int TN_NACC = 2;            // accumulators
-constexpr int TN_TMEM_COLS = TN_NACC * TN_CB;
 static_assert(TN_TEAMS == 1 || TN_TEAMS == TN_NACC, "a team owns an accumulator, or one team takes them in turn");
 
-template <int M>
+// GS = 0 stands for the tile-size-only constants (the constant matrix).  A work item covers one group
+// of 64, 128 or 256 channels (NB boxes of 64 channels per tile, side by side in the accumulator), or
+// two groups of 32.
+template <int M, int GS = 64>
 struct TnCfg {
+    static constexpr int NB = GS > 64 ? GS / 64 : 1;          // boxes of 64 channels per tile
+    static constexpr int ACC_COLS = NB * TN_CB;               // channels per work item = accumulator columns
+    static constexpr int TMEM_COLS = TN_NACC * ACC_COLS;      // 128, 256 or 512
+    static constexpr int NSTRIP = NB == 1 ? 3 : 2;
+    static constexpr int CTAS_PER_SM = NB == 4 ? 1 : 2;       // by shared memory and (groups of 256) tensor memory
     static constexpr int NN = M + 2;
     static constexpr int P = NN * NN;
     static constexpr int TB = M == 6 ? 2 : 3;                 // tiles per work item
@@ -62,13 +75,13 @@ struct TnCfg {
     static constexpr int A_BYTES = (A_ROWS * 128 + 1023) / 1024 * 1024;   // rows of 64 fp16, 128-byte swizzle
     static constexpr int AMAT_BYTES = PL * 128;               // the matrix itself
     static constexpr int BOX_BYTES = NN * 8 * 128;            // one tile's box
-    static constexpr int STRIP_BYTES = TB * BOX_BYTES;
-    static constexpr size_t SMEM_BYTES = 1024 + A_BYTES + TN_NSTRIP * STRIP_BYTES;
+    static constexpr int STRIP_BYTES = TB * NB * BOX_BYTES;
+    static constexpr size_t SMEM_BYTES = 1024 + A_BYTES + NSTRIP * STRIP_BYTES;
 };
 
 struct TnShared {
-    uint64_t strip_full[TN_NSTRIP];
-    uint64_t strip_empty[TN_NSTRIP];
+    uint64_t strip_full[TN_MAX_NSTRIP];
+    uint64_t strip_empty[TN_MAX_NSTRIP];
     uint64_t acc_full[TN_NACC];
     uint64_t acc_empty[TN_NACC];
     uint32_t tmem_base;
@@ -89,7 +102,8 @@ template <int M, int GS>
 __global__ void __launch_bounds__(TN_THREADS, 2)
 input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Geometry g, ScaleTables tab)
 {
-    using C = TnCfg<M>;
+    using C = TnCfg<M, GS>;
+    constexpr int TN_NSTRIP = C::NSTRIP;
     extern __shared__ unsigned char smem_dyn[];
     __shared__ TnShared sh;
     unsigned char *base = reinterpret_cast<unsigned char *>(
@@ -121,7 +135,7 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
         asm volatile("griddepcontrol.wait;" ::: "memory");
     } else {
         if (warp == 1) {
-            ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TN_TMEM_COLS);
+            ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), C::TMEM_COLS);
             ptx::tmem_relinquish();
         }
         // the A operand: zero rows, the constant matrix (a plain copy; it does not depend on the previous
@@ -158,8 +172,11 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
                 ptx::mbar_arrive_expect_tx(bar, (uint32_t)C::STRIP_BYTES);
 #pragma unroll
                 for (int tl = 0; tl < C::TB; ++tl)
-                    ptx::tma_load_4d(ptx::smem_u32(strips + sb * C::STRIP_BYTES + tl * C::BOX_BYTES), &tmx, bar,
-                                     cblk * TN_CB, (chunk * C::TB + tl) * M - 1, th * M - 1, img);
+#pragma unroll
+                    for (int nb = 0; nb < C::NB; ++nb)
+                        ptx::tma_load_4d(
+                            ptx::smem_u32(strips + sb * C::STRIP_BYTES + (tl * C::NB + nb) * C::BOX_BYTES), &tmx, bar,
+                            cblk * C::ACC_COLS + nb * TN_CB, (chunk * C::TB + tl) * M - 1, th * M - 1, img);
             }
             __syncwarp();
             ++issued;
@@ -190,18 +207,22 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
                 break;
             ptx::tc_fence_after();
             if (lane == 0) {
-                const uint32_t d = tmem_base + (uint32_t)(slot * TN_CB);
                 const uint32_t b_lo = s_lo0 + (uint32_t)((sb * C::STRIP_BYTES) >> 4);
 #pragma unroll
-                for (int tl = 0; tl < C::TB; ++tl)
+                for (int nb = 0; nb < C::NB; ++nb) {              // 64 accumulator columns per box of channels
+                    const uint32_t d = tmem_base + (uint32_t)(slot * C::ACC_COLS + nb * TN_CB);
 #pragma unroll
-                    for (int ks = 0; ks < C::KSTEPS; ++ks) {
-                        // the matrix's rows land on accumulator rows tl * PL ...: start tl * PL rows early
-                        const uint32_t al = a_lo0 + (uint32_t)(((C::Z0 - tl * C::PL) * 128 + ks * 32) >> 4);
-                        const uint32_t bl = b_lo + (uint32_t)((tl * C::BOX_BYTES + ks * 2048) >> 4);
-                        if (tl == 0 && ks == 0) ptx::umma_f16_lo<false>(d, al, bl, dhi, idesc);
-                        else ptx::umma_f16_lo<true>(d, al, bl, dhi, idesc);
-                    }
+                    for (int tl = 0; tl < C::TB; ++tl)
+#pragma unroll
+                        for (int ks = 0; ks < C::KSTEPS; ++ks) {
+                            // the matrix's rows land on accumulator rows tl * PL ...: start tl * PL rows early
+                            const uint32_t al = a_lo0 + (uint32_t)(((C::Z0 - tl * C::PL) * 128 + ks * 32) >> 4);
+                            const uint32_t bl =
+                                b_lo + (uint32_t)(((tl * C::NB + nb) * C::BOX_BYTES + ks * 2048) >> 4);
+                            if (tl == 0 && ks == 0) ptx::umma_f16_lo<false>(d, al, bl, dhi, idesc);
+                            else ptx::umma_f16_lo<true>(d, al, bl, dhi, idesc);
+                        }
+                }
                 ptx::umma_commit(ptx::smem_u32(&sh.acc_full[slot]));
                 ptx::umma_commit(ptx::smem_u32(&sh.strip_empty[sb]));
             }
@@ -229,8 +250,8 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
             const int tw = chunk * C::TB + tl;
             const bool valid = row_ok && tw < g.TW;
             const int t = srow * g.TW + tw;
-            const uint32_t taddr = taddr0 + (uint32_t)(slot * TN_CB);
-            int8_t *dst = a.Xq + ((size_t)p * g.T + t) * g.C + cblk * TN_CB;
+            const uint32_t taddr = taddr0 + (uint32_t)(slot * C::ACC_COLS);
+            int8_t *dst = a.Xq + ((size_t)p * g.T + t) * g.C + cblk * C::ACC_COLS;
             uint32_t v[32];
             if (GS == 32) {
                 float *sd = a.sX + ((size_t)p * g.G + cblk * 2) * g.Ts + t;
@@ -249,6 +270,30 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
                         codes32(v, sp, sl, inv, dst + 32 * h);
                         sd[(size_t)h * g.Ts] = scale;
                     }
+                }
+            } else if (GS > 64) {
+                // a group of 128 or 256 channels: abs-max over all its columns, then every 32 columns
+                // again from TMEM for the codes
+                float m = 0.f;
+#pragma unroll
+                for (int c = 0; c < C::ACC_COLS / 32; ++c) {
+                    ptx::tmem_ld_x32(taddr + (uint32_t)(32 * c), v);
+                    ptx::tmem_ld_wait();
+                    m = absmax32(v, m);
+                }
+                float scale, inv;
+                group_scale_inv(fabsf(scaled(m, sp, sl)), scale, inv);
+                if (valid) a.sX[((size_t)p * g.G + cblk) * g.Ts + t] = scale;
+#pragma unroll
+                for (int c = 0; c < C::ACC_COLS / 32; ++c) {
+                    ptx::tmem_ld_x32(taddr + (uint32_t)(32 * c), v);
+                    ptx::tmem_ld_wait();
+                    if (c == C::ACC_COLS / 32 - 1) {
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.acc_empty[slot]));
+                    }
+                    if (valid) codes32(v, sp, sl, inv, dst + 32 * c);
                 }
             } else {
                 // abs-max over both halves, codes for the second half from the registers, then the
@@ -283,7 +328,7 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, TN_TMEM_COLS);
+        ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
 }
 
@@ -325,7 +370,7 @@ void *g_tn_amat[kTnMaxDevices][2];
 template <int M, int GS>
 cudaError_t launch_tn(const wfq_plan &plan, cudaStream_t stream)
 {
-    using C = TnCfg<M>;
+    using C = TnCfg<M, GS>;
     const Geometry &g = plan.geo;
     TnArgs a;
     a.Xq = plan.ws.Xq;
@@ -334,11 +379,11 @@ cudaError_t launch_tn(const wfq_plan &plan, cudaStream_t stream)
     a.wait_cycles = plan.wait_cycles;
     a.amat = static_cast<const uint4 *>(g_tn_amat[plan.device][M == 6 ? 1 : 0]);
     a.NCH = (g.TW + C::TB - 1) / C::TB;
-    a.NCB = g.C / TN_CB;
+    a.NCB = g.C / C::ACC_COLS;
     a.items = g.N * g.TH * a.NCH * a.NCB;
     a.debug_skip_item = plan.debug_skip_item;
     if (!a.amat) return cudaErrorInvalidValue;
-    const int slots = 2 * plan.sm_count;
+    const int slots = C::CTAS_PER_SM * plan.sm_count;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(a.items < slots ? a.items : slots));
     cfg.blockDim = dim3(TN_THREADS);
@@ -354,12 +399,12 @@ cudaError_t launch_tn(const wfq_plan &plan, cudaStream_t stream)
 
 }  // namespace
 
-// Does the tensor-core NHWC kernel serve this plan?  fp16, groups of 32 or 64, channels in blocks of 64,
-// the paper's two tile sizes.
+// Does the tensor-core NHWC kernel serve this plan?  fp16, groups of 32, 64, 128 or 256, channels in blocks
+// of 64, the paper's two tile sizes.
 bool input_transform_tcn_applies(const wfq_plan &plan)
 {
     const Geometry &g = plan.geo;
-    return plan.in_dtype == WFQ_F16 && (g.gs == 32 || g.gs == 64) && g.C % TN_CB == 0 && (g.m == 4 || g.m == 6);
+    return plan.in_dtype == WFQ_F16 && (g.gs == 32 || g.gs == 64 || g.gs == 128 || g.gs == 256) && g.C % TN_CB == 0 && (g.m == 4 || g.m == 6);
 }
 
 // Box of the input tensor map for this kernel: {64 channels, 8 columns, n rows, 1 image}, 128-byte swizzle.
@@ -378,10 +423,14 @@ cudaError_t setup_input_transform_tcn()
     auto attr = [](auto kern, size_t smem) {
         return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     };
-    if ((e = attr(input_transform_tcn_kernel<4, 32>, TnCfg<4>::SMEM_BYTES)) != cudaSuccess) return e;
-    if ((e = attr(input_transform_tcn_kernel<4, 64>, TnCfg<4>::SMEM_BYTES)) != cudaSuccess) return e;
-    if ((e = attr(input_transform_tcn_kernel<6, 32>, TnCfg<6>::SMEM_BYTES)) != cudaSuccess) return e;
-    if ((e = attr(input_transform_tcn_kernel<6, 64>, TnCfg<6>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = attr(input_transform_tcn_kernel<4, 32>, TnCfg<4, 32>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = attr(input_transform_tcn_kernel<4, 64>, TnCfg<4, 64>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = attr(input_transform_tcn_kernel<4, 128>, TnCfg<4, 128>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = attr(input_transform_tcn_kernel<4, 256>, TnCfg<4, 256>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = attr(input_transform_tcn_kernel<6, 32>, TnCfg<6, 32>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = attr(input_transform_tcn_kernel<6, 64>, TnCfg<6, 64>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = attr(input_transform_tcn_kernel<6, 128>, TnCfg<6, 128>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = attr(input_transform_tcn_kernel<6, 256>, TnCfg<6, 256>::SMEM_BYTES)) != cudaSuccess) return e;
     if (!g_tn_amat[dev][0]) {
         std::vector<uint16_t> a4, a6;
         build_amat<4>(a4);
@@ -399,9 +448,12 @@ cudaError_t setup_input_transform_tcn()
 
 cudaError_t launch_input_transform_tcn(const wfq_plan &plan, cudaStream_t stream)
 {
+    const int gs = plan.geo.gs;
     if (plan.geo.m == 4)
-        return plan.geo.gs == 32 ? launch_tn<4, 32>(plan, stream) : launch_tn<4, 64>(plan, stream);
-    return plan.geo.gs == 32 ? launch_tn<6, 32>(plan, stream) : launch_tn<6, 64>(plan, stream);
+        return gs == 32 ? launch_tn<4, 32>(plan, stream) : gs == 64 ? launch_tn<4, 64>(plan, stream)
+             : gs == 128 ? launch_tn<4, 128>(plan, stream) : launch_tn<4, 256>(plan, stream);
+    return gs == 32 ? launch_tn<6, 32>(plan, stream) : gs == 64 ? launch_tn<6, 64>(plan, stream)
+         : gs == 128 ? launch_tn<6, 128>(plan, stream) : launch_tn<6, 256>(plan, stream);
 }
 
 }  // namespace wfq

@@ -228,6 +228,9 @@ def test_contraction_shapes_agree(layer):
     Layer(9, 128, 32, 7, 7, 6, 64, "f16", "relu_heavy", "kaiming", 9, 8, 10),
     Layer(2, 64, 32, 5, 5, 4, 32, "f16", "silu_outlier", "kaiming_chan", 9, 8, 11),
     Layer(3, 128, 40, 30, 18, 6, 32, "f16", "silu_outlier", "kaiming_chan", 9, 8, 12),
+    # tensor cores, groups of 128 and 256 (two and four boxes of channels per tile), the other tile size each
+    Layer(2, 256, 32, 22, 20, 4, 128, "f16", "silu_outlier", "kaiming_chan", 9, 8, 13),
+    Layer(1, 512, 32, 20, 26, 6, 256, "f16", "silu_outlier", "kaiming_chan", 9, 8, 14),
 ], ids=lambda L: L.name)
 def test_nhwc_input_matches_nchw(layer):
     """x given as [N][H][W][C].  With the plain NHWC kernel (TMA-staged strips, debug option 1) the
