@@ -780,6 +780,19 @@ def run_wfq(args):
                 per_config[f"cfg{cfg}"] = s2
                 del w2
                 torch.cuda.empty_cache()
+                if cfg in (2, 3, 4) and not args.no_extras:      # the same layers handed over as NHWC
+                    w2 = Workload(cfg, None, dev, stream, flush, use_graph=not args.no_graph, nhwc=True)
+                    for _ in range(3):
+                        flush.zero_()
+                        w2.step()
+                    torch.cuda.synchronize(dev)
+                    ms = [statistics.median(w2.timed_replays(reps)) for _ in range(10)]
+                    s2n, _, _ = w2.summary(statistics.mean(ms), w2.kernel_split(10), peak)
+                    s2["nhwc_input"] = {"value": s2n["value"], "unit": UNIT, "us_per_step": s2n["us_per_step"],
+                                        "input_transform_us_per_step": s2n["kernels"][KERNELS[0]]["us_per_step"]}
+                    w2.close()
+                    del w2
+                    torch.cuda.empty_cache()
             except Exception as exc:
                 per_config[f"cfg{cfg}"] = {"error": repr(exc)}
 
