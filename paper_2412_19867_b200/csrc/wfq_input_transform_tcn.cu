@@ -44,15 +44,10 @@
 namespace wfq {
 namespace {
 
-// quantizer teams of four warps; team k takes the CTA's items k, k + TEAMS, ...  (a second team, one per
-// accumulator, and a fourth strip were measured: no difference on any configured layer)
-constexpr int TN_TEAMS = 1;
-constexpr int TN_FIRST_QUANT = 4;
-constexpr int TN_THREADS = 32 * (TN_FIRST_QUANT + 4 * TN_TEAMS);
+constexpr int TN_FIRST_QUANT = 4;   // warps 0-3: producer, MMA issuer, two idle; then the quantizer teams of four warps
 constexpr int TN_CB = 64;             // channels per box = N of one MMA
 constexpr int TN_MAX_NSTRIP = 3;      // strip ring (at most)
-constexpr int TN_NACC = 2;            // accumulators
-static_assert(TN_TEAMS == 1 || TN_TEAMS == TN_NACC, "a team owns an accumulator, or one team takes them in turn");
+constexpr int TN_MAX_NACC = 4;        // accumulators (at most)
 
 // GS = 0 stands for the tile-size-only constants (the constant matrix).  A work item covers one group
 // of 64, 128 or 256 channels (NB boxes of 64 channels per tile, side by side in the accumulator), or
@@ -61,7 +56,16 @@ template <int M, int GS = 64>
 struct TnCfg {
     static constexpr int NB = GS > 64 ? GS / 64 : 1;          // boxes of 64 channels per tile
     static constexpr int ACC_COLS = NB * TN_CB;               // channels per work item = accumulator columns
-    static constexpr int TMEM_COLS = TN_NACC * ACC_COLS;      // 128, 256 or 512
+    // Two accumulators and one quantizer team of four warps.  The code takes NACC accumulators and TEAMS
+    // teams (team k quantizes the CTA's items k, k + TEAMS, ...); four accumulators with two teams and a
+    // fourth strip were measured and change nothing: per-CTA timestamps show a box arriving every 1.3 us
+    // whatever the number in flight (the boxes of the two CTAs of an SM arrive at about 28 KB/us, 4 TB/s
+    // over the chip, three times the unique input bytes because neighbouring tiles' boxes overlap), with
+    // the MMA issuer and the quantizers waiting for them.
+    static constexpr int NACC = 2;
+    static constexpr int TEAMS = 1;
+    static constexpr int THREADS = 32 * (TN_FIRST_QUANT + 4 * TEAMS);
+    static constexpr int TMEM_COLS = NACC * ACC_COLS;         // 128, 256 or 512
     static constexpr int NSTRIP = NB == 1 ? 3 : 2;
     static constexpr int CTAS_PER_SM = NB == 4 ? 1 : 2;       // by shared memory and (groups of 256) tensor memory
     static constexpr int NN = M + 2;
@@ -82,8 +86,8 @@ struct TnCfg {
 struct TnShared {
     uint64_t strip_full[TN_MAX_NSTRIP];
     uint64_t strip_empty[TN_MAX_NSTRIP];
-    uint64_t acc_full[TN_NACC];
-    uint64_t acc_empty[TN_NACC];
+    uint64_t acc_full[TN_MAX_NACC];
+    uint64_t acc_empty[TN_MAX_NACC];
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -99,11 +103,11 @@ struct TnArgs {
 };
 
 template <int M, int GS>
-__global__ void __launch_bounds__(TN_THREADS, 2)
+__global__ void __launch_bounds__((TnCfg<M, GS>::THREADS), 2)
 input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Geometry g, ScaleTables tab)
 {
     using C = TnCfg<M, GS>;
-    constexpr int TN_NSTRIP = C::NSTRIP;
+    constexpr int TN_NSTRIP = C::NSTRIP, TN_NACC = C::NACC, TN_TEAMS = C::TEAMS, TN_THREADS = C::THREADS;
     extern __shared__ unsigned char smem_dyn[];
     __shared__ TnShared sh;
     unsigned char *base = reinterpret_cast<unsigned char *>(
@@ -239,10 +243,12 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
         const float sp = row_ok ? tab.in_scale[p] : 0.f, sl = row_ok ? tab.in_scale_lo[p] : 0.f;
         const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16);
         // one team: both accumulators in turn; two teams: team k owns accumulator k
+        // the CTA's j-th item uses accumulator j % NACC; team k takes j = k, k + TEAMS, ...
         const int team = (warp - TN_FIRST_QUANT) >> 2;
-        int slot = TN_TEAMS == 1 ? 0 : team;
-        uint32_t aphase = 0;
-        for (int item = blockIdx.x + team * stride; item < a.items; item += TN_TEAMS * stride) {
+        int j = team;
+        for (int item = blockIdx.x + team * stride; item < a.items; item += TN_TEAMS * stride, j += TN_TEAMS) {
+            const int slot = j % TN_NACC;
+            const uint32_t aphase = (uint32_t)(j / TN_NACC) & 1u;
             if (!wait_bounded(ptx::smem_u32(&sh.acc_full[slot]), aphase, ctx, kWaitAccFull)) break;
             ptx::tc_fence_after();
             const int cblk = item % a.NCB, rest = item / a.NCB;
@@ -316,11 +322,6 @@ input_transform_tcn_kernel(const __grid_constant__ CUtensorMap tmx, TnArgs a, Ge
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.acc_empty[slot]));
                 if (valid) codes32(v, sp, sl, inv, dst);
             }
-            if (TN_TEAMS == 1) {
-                if (++slot == TN_NACC) { slot = 0; aphase ^= 1u; }
-            } else {
-                aphase ^= 1u;
-            }
         }
     }
 
@@ -386,7 +387,7 @@ cudaError_t launch_tn(const wfq_plan &plan, cudaStream_t stream)
     const int slots = C::CTAS_PER_SM * plan.sm_count;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(a.items < slots ? a.items : slots));
-    cfg.blockDim = dim3(TN_THREADS);
+    cfg.blockDim = dim3(C::THREADS);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
