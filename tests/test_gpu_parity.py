@@ -446,6 +446,17 @@ def test_host_buffer_entry_point_in_chunks_matches_device_one():
         conv.forward_host(xh, yh)
         assert torch.equal(yh, y_dev)
     conv.check_status()
+    # the same batch handed over as NHWC (tensor-core input transform in the chunks' plans) with bf16 output
+    conv.set_input_layout("nhwc")
+    conv.set_output_dtype("bf16")
+    xn = xd.permute(0, 2, 3, 1).contiguous()
+    y_dev = conv.forward(xn).cpu()
+    xnh = xn.cpu().pin_memory()
+    for _ in range(2):
+        yh = torch.zeros(y_dev.shape, dtype=torch.bfloat16).pin_memory()
+        conv.forward_host(xnh, yh)
+        assert torch.equal(yh, y_dev)
+    conv.check_status()
     conv.close()
 
 
