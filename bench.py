@@ -283,17 +283,20 @@ class Workload:
     """The layers of one configuration: plans, device tensors, and the step as a CUDA graph."""
 
     def __init__(self, cfg, only_layer, dev, stream, flush, use_graph=True, k1_kernel=0, full_quant=None,
-                 nhwc=False, streams=1):
+                 nhwc=False, streams=1, w_bits=8):
         import torch
         from paper_2412_19867_b200 import binding as b
         from paper_2412_19867_b200 import workloads as wl
         self.torch, self.b, self.dev, self.stream, self.flush = torch, b, dev, stream, flush
         self.cfg = cfg
+        self.w_bits = w_bits
         self.layers = select_layers(wl, cfg, only_layer)
         self.tensors = [wl.make_tensors(L) for L in self.layers]
         self.convs, self.xs, self.ys = [], [], []
         for L, (x, w, sB, sG) in zip(self.layers, self.tensors):
             conv = b.Conv(L.N, L.C, L.K, L.H, L.W, L.m, L.gs, L.dtype, dev)
+            if w_bits != 8:                 # filter codes in [-7, 7]; activations stay at 8 bits
+                conv.set_weight_bits(w_bits)
             conv.prepare(torch.from_numpy(w).to(dev), list(sB), list(sG))
             if k1_kernel:
                 b.wfq_plan_set_debug_option(conv.plan, b.WFQ_DEBUG_INPUT_TRANSFORM_KERNEL, k1_kernel)
@@ -450,7 +453,10 @@ class Workload:
             T = conv.T
             tiles = np.unique(np.concatenate([[0, T - 1], rng.integers(0, T, tiles_per_layer)]))
             ks = np.unique(np.concatenate([[0, L.K - 1], rng.integers(0, L.K, channels)]))
-            ref = orc.wfq(x, w[ks], L.m, L.gs, sB=sB, sG=sG, tiles=tiles)
+            filters = None
+            if self.w_bits != 8:
+                filters = orc.prepare_filters(w[ks], L.m, L.gs, orc.matrices(L.m, sB, sG, None), bits=self.w_bits)
+            ref = orc.wfq(x, w[ks], L.m, L.gs, sB=sB, sG=sG, tiles=tiles, filters=filters)
             xq = conv.buffer(b.WFQ_BUF_XQ)[:, torch.from_numpy(tiles).to(self.dev)].cpu().numpy()
             mism += int(np.count_nonzero(xq != ref.Xq))
             ncodes += xq.size
@@ -850,6 +856,31 @@ def run_wfq(args):
         except Exception as exc:
             nhwc = {"error": repr(exc)}
 
+    # ---- 4-bit filter codes (W4A8) on the UNet block, reported beside ----
+    w4 = None
+    if rank == 0 and world == 1 and not args.no_extras and args.only_layer is None:
+        try:
+            w6 = Workload(4, None, dev, stream, flush, use_graph=not args.no_graph, w_bits=4)
+            for _ in range(3):
+                flush.zero_()
+                w6.step()
+            torch.cuda.synchronize(dev)
+            ms = statistics.mean(statistics.median(w6.timed_replays(reps)) for _ in range(10))
+            flush.zero_()
+            w6.step()
+            torch.cuda.synchronize(dev)
+            w4 = {"workload": "cfg4 with the filters quantized to 4 bits (codes in [-7, 7], one per byte on the "
+                              "device; activations at 8 bits)",
+                  "value": w6.step_ops / (ms * 1e-3) / 1e12, "unit": UNIT, "us_per_step": ms * 1e3,
+                  "parity": w6.parity(),
+                  "filter_blob_bytes": int(sum(b.wfq_filters_bytes(c.plan) for c in w6.convs)),
+                  "note": "same kernels as with 8-bit filters; the exported filter blob stores two codes per byte"}
+            w6.close()
+            del w6
+            torch.cuda.empty_cache()
+        except Exception as exc:
+            w4 = {"error": repr(exc)}
+
     # ---- the headline workload with its layers on three streams, reported beside ----
     concurrent = None
     if rank == 0 and world == 1 and not args.no_extras and args.only_layer is None:
@@ -892,7 +923,7 @@ def run_wfq(args):
                            "parallelism": "replicas" if world > 1 else "single GPU"},
                 "timing": timing, "us_per_layer": head["us_per_layer"], "wall_s_timed_region": wall,
                 "warm": warm, "sustained": sustained, "roofline": roofline, "contraction": contraction,
-                "parity": parity, "per_config": per_config, "full_quant": full_quant, "nhwc_input": nhwc, "layers_on_three_streams": concurrent, "cpu_baseline": cpu, "e2e": e2e,
+                "parity": parity, "per_config": per_config, "full_quant": full_quant, "nhwc_input": nhwc, "layers_on_three_streams": concurrent, "w4_weights": w4, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": 3 * len(layers) * args.steps * reps, "clocks": clocks}
         print(json.dumps(line), flush=True)
     if world > 1:
