@@ -283,7 +283,8 @@ wfq_status_t wfq_conv_forward(wfq_plan_t *plan, const void *x_dev, float *y_dev,
  *                       prepared plan; synchronous with respect to `stream`
  *   wfq_filters_import  makes the plan prepared from a blob written for the same C, K, tile and
  *                       group size (WFQ_ERR_INVALID_ARG otherwise, plan unchanged); the plan takes
- *                       the blob's weight bit width; the blob is copied before the call returns
+ *                       the blob's weight bit width; the blob is copied before the call returns;
+ *                       a CUDA error during the copy (WFQ_ERR_CUDA) leaves the plan unprepared
  */
 size_t wfq_filters_bytes(const wfq_plan_t *plan);
 wfq_status_t wfq_filters_export(wfq_plan_t *plan, void *host_buf, size_t bytes, void *stream);

@@ -446,6 +446,8 @@ wfq_status_t wfq_filters_import(wfq_plan_t *plan, const void *host_buf, size_t b
     cudaStream_t st = as_stream(stream);
     wfq_status_t bs = ensure_filter_buffers(plan, st);
     if (bs != WFQ_OK) return bs;
+    // from here on the plan's filters are being replaced: a CUDA error below leaves it unprepared
+    plan->prepared = false;
     for (int i = 0; i < g.n; ++i) { plan->sB[i] = h.sB[i]; plan->sG[i] = h.sG[i]; plan->sA[i] = h.sA[i]; }
     fill_scale_tables(plan);
     plan->w_bits = w_bits;
