@@ -27,8 +27,10 @@
 //   warp 0     TMA producer: per work item TB boxes (one per tile; tiles past the end of the tile
 //              row are loaded all the same and come back as zeros) into a ring of three strips (two for
 //              groups of 128 and 256)
-//   warp 1     owns TMEM; one lane issues TB * n / 2 MMAs per item (M = 128, N = 64, K = 16) into one
-//              of two accumulators of 64 columns, commits the accumulator and the strip
+//   warp 1     owns TMEM; one lane issues TB * n / 2 MMAs per box of channels (M = 128, N = 64, K = 16) into
+//              one of two accumulators of 64, 128 or 256 columns, commits the accumulator and the strip
+//   (warp 0 starts its first boxes right after the barrier initialisation; warps 1-7 meanwhile allocate
+//   TMEM and build the A operand and meet at a named barrier of their own)
 //   warps 4-7  quantizers: warp % 4 selects the 32 TMEM lanes; per-position factor, abs-max, scale,
 //              codes, one 32-byte store per 32 codes
 // All waits are bounded; on expiry the CTA records the wait, drains its copies and frees TMEM.
